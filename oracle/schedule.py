@@ -1,15 +1,15 @@
 """Batching analysis, the slow and obvious way.  TEST INFRASTRUCTURE ONLY.
 
-The paper files every recorded computation node in a table "according to their
-depth", notes that nodes of one depth are independent of each other, and runs
-the table in depth order (Section 4.2).  For a forest of Tree-LSTM cells the
+The paper files every recorded computation node in a table keyed by the node's
+depth, observes that no node of a depth depends on another node of that depth,
+and runs the table in depth order (Section 4.2).  For a forest of Tree-LSTM cells the
 computation node of tree node v consumes the results of v's children, so its
 depth is its height above the leaves:
 
     depth(v) = 0                         if v has no children
     depth(v) = 1 + max_k depth(child_k)  otherwise
 
-and the table is (Section 4.3, "reside in the same slot"):
+and the table is (Section 4.3: nodes that can be batched share one slot):
 
     level_ptr[d] = number of nodes with depth < d,   d = 0 .. n_levels
     perm         = node ids ordered by (depth, id)

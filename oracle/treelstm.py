@@ -26,7 +26,10 @@ in fp64, so that rounding can be told apart from a mistake.
 ``quantize="bf16_edges"`` is the same for an evaluation that takes the child sum
 behind the product, U_iou h~_j = sum_k U_iou h_k: the only recurrent GEMM operand is
 then h_k, so each h_k is rounded and the sum of the rounded rows is not rounded again.
-The paper fixes no precision; both are bf16-GEMM evaluations of the same cell.
+``quantize="bf16_rows"`` is the evaluation that keeps only a bf16 copy of every h_k for
+the recurrence: the child sum is taken over the rounded rows and, being a GEMM operand
+itself, is rounded once more, h~_j = bf16(sum_k bf16(h_k)).
+The paper fixes no precision; all three are bf16-GEMM evaluations of the same cell.
 
 Nothing here is shared with the CUDA path.  Pins: tests/test_oracle_treelstm.py.
 """
@@ -84,7 +87,7 @@ def forward(child_ptr, child_idx, x, W, U, b, roots=None, quantize=None, x_of=No
     H = U.shape[1]
     assert W.shape[0] == 4 * H and U.shape[0] == 4 * H and b.shape[0] == 4 * H
     q = (lambda a: a) if quantize is None else bf16_round
-    if quantize not in (None, "bf16", "bf16_edges"):
+    if quantize not in (None, "bf16", "bf16_edges", "bf16_rows"):
         raise ValueError(quantize)
     W = q(W)
     U = q(U)
@@ -103,10 +106,12 @@ def forward(child_ptr, child_idx, x, W, U, b, roots=None, quantize=None, x_of=No
             h_sum = h_sum + h[k]
         z = W @ xj + b
         z_i, z_o, z_u, z_f = z[0:H], z[H:2 * H], z[2 * H:3 * H], z[3 * H:4 * H]
-        if quantize == "bf16_edges":
+        if quantize in ("bf16_edges", "bf16_rows"):
             hs = np.zeros(H, dtype=np.float64)
             for k in kids:
                 hs = hs + q(h[k])
+            if quantize == "bf16_rows":
+                hs = q(hs)
         else:
             hs = q(h_sum)
         i = sigmoid(z_i + U_i @ hs)

@@ -212,3 +212,88 @@ def test_x_of_callback_equals_array():
     h, c = ot.forward(f.child_ptr, f.child_idx, _x(w), w.W, w.U, w.b)
     h2, c2 = ot.forward(f.child_ptr, f.child_idx, None, w.W, w.U, w.b, x_of=lambda v: w.table[w.token[v]])
     assert np.array_equal(h, h2) and np.array_equal(c, c2)
+
+
+# ---- where the bf16-matched modes round -----------------------------------------------------------------
+# A scalar cell (D = H = 1) over one root with two different leaves, worked with math.exp.  Every rounded value is
+# typed here as a literal; that a literal is THE bfloat16 neighbour of the value it stands for is checked from the
+# format's definition (8 significant bits, within half a unit in the last place), not with the checker's routine.
+def _is_bf16(v):
+    m, _ = math.frexp(v)
+    return float(m * 256.0).is_integer()
+
+
+def _is_nearest_bf16(v, lit):
+    _, e = math.frexp(v)                       # |v| in [2^(e-1), 2^e): one unit in the last place is 2^(e-8)
+    half = 2.0 ** (e - 9)
+    m, _ = math.frexp(lit)
+    even = int(abs(m) * 256.0) % 2 == 0        # a value half-way between two neighbours goes to the even one
+    return _is_bf16(lit) and (abs(v - lit) < half or (abs(v - lit) == half and even))
+
+
+_RX = [0.5029296875, 0.28271484375, 1.0341796875]                      # x of root, leaf 1, leaf 2
+_RW = [0.301513671875, -0.70263671875, 1.10498046875, 0.40087890625]  # i, o, u, f
+_RU = [-0.200439453125, 0.90185546875, 0.60107421875, -1.3076171875]
+_RB = [0.05, -0.1, 0.2, 0.3]                                          # the bias is never rounded
+_RXQ = [0.50390625, 0.283203125, 1.03125]
+_RWQ = [0.30078125, -0.703125, 1.1015625, 0.400390625]
+_RUQ = [-0.2001953125, 0.90234375, 0.6015625, -1.3046875]
+# bfloat16 neighbours of the leaves' h computed from the rounded inputs (h_1 = 0.104938..., h_2 = 0.143876...), of their
+# sum (0.248814...), and of the sum of the two rounded rows (0.24853515625, half-way between two neighbours)
+_RH1Q, _RH2Q, _RHSUMQ, _RHROWSQ = 0.10498046875, 0.1435546875, 0.2490234375, 0.248046875
+
+
+def _rounding_chain(mode, drop=None):
+    """(h_root, c_root, h_1, h_2) of the scalar cell, with the roundings of `mode` minus the one named by `drop`."""
+    r = lambda name, raw, rounded: raw if (mode is None or drop == name) else rounded
+    x = [r("x", a, b) for a, b in zip(_RX, _RXQ)]
+    W = [r("W", a, b) for a, b in zip(_RW, _RWQ)]
+    U = [r("U", a, b) for a, b in zip(_RU, _RUQ)]
+
+    def leaf(xv):
+        cc = _sig(W[0] * xv + _RB[0]) * math.tanh(W[2] * xv + _RB[2])
+        return _sig(W[1] * xv + _RB[1]) * math.tanh(cc), cc
+
+    (h1, c1), (h2, c2) = leaf(x[1]), leaf(x[2])
+    if mode is not None and drop is None:
+        assert _is_nearest_bf16(h1, _RH1Q) and _is_nearest_bf16(h2, _RH2Q) and _is_nearest_bf16(h1 + h2, _RHSUMQ)
+        assert _is_nearest_bf16(_RH1Q + _RH2Q, _RHROWSQ) and _RH1Q + _RH2Q != _RHROWSQ
+    h1q, h2q = r("h_k", h1, _RH1Q), r("h_k", h2, _RH2Q)
+    if mode == "bf16":
+        hs = r("h_sum", h1 + h2, _RHSUMQ)        # the child sum of the exact rows, rounded once
+    elif mode == "bf16_edges":
+        hs = h1q + h2q                            # the rounded rows, added exactly
+    elif mode == "bf16_rows":
+        hs = r("h_sum", h1q + h2q, _RHROWSQ)      # the rounded rows, added exactly, the sum rounded again
+    else:
+        hs = h1 + h2
+    i = _sig(W[0] * x[0] + _RB[0] + U[0] * hs)
+    o = _sig(W[1] * x[0] + _RB[1] + U[1] * hs)
+    u = math.tanh(W[2] * x[0] + _RB[2] + U[2] * hs)
+    f1 = _sig(W[3] * x[0] + _RB[3] + U[3] * h1q)
+    f2 = _sig(W[3] * x[0] + _RB[3] + U[3] * h2q)
+    c0 = i * u + f1 * c1 + f2 * c2                # c_k is state: never rounded
+    return o * math.tanh(c0), c0, h1, h2
+
+
+@pytest.mark.parametrize("mode", [None, "bf16", "bf16_edges", "bf16_rows"])
+def test_rounding_points_of_the_matched_modes_by_hand(mode):
+    for raw, lit in zip(_RX + _RW + _RU, _RXQ + _RWQ + _RUQ):
+        assert raw != lit and _is_nearest_bf16(raw, lit)
+    f = wl.forest_from_parents([np.array([-1, 0, 0])])
+    h, c = ot.forward(f.child_ptr, f.child_idx, np.array(_RX).reshape(3, 1), np.array(_RW).reshape(4, 1),
+                      np.array(_RU).reshape(4, 1), np.array(_RB), quantize=mode)
+    h0, c0, h1, h2 = _rounding_chain(mode)
+    assert abs(h[0, 0] - h0) < 1e-15 and abs(c[0, 0] - c0) < 1e-15
+    assert abs(h[1, 0] - h1) < 1e-15 and abs(h[2, 0] - h2) < 1e-15
+    if mode is None:
+        return
+    # a checker that forgot any one of the roundings would land on one of these chains instead: each is far away
+    points = ["x", "W", "U", "h_k"] + (["h_sum"] if mode != "bf16_edges" else [])
+    for drop in points:
+        hd, cd, _, _ = _rounding_chain(mode, drop)
+        assert max(abs(hd - h[0, 0]), abs(cd - c[0, 0])) > 2e-6, drop
+    # and the two modes differ from each other and from the plain evaluation
+    for other in {"bf16", "bf16_edges", "bf16_rows"} - {mode}:
+        assert abs(_rounding_chain(other)[0] - h0) > 1e-6, other
+    assert abs(_rounding_chain(None)[0] - h0) > 1e-4
