@@ -2,7 +2,8 @@
 
     python bench.py --gpus N --steps K --warmup W [--config 1..5] [--impl reference]
 
-Prints ONE JSON line (rank 0).  Inputs are seeded synthetic forests (workloads.py).  `value` is nodes/s
+With N > 1 and no WORLD_SIZE in the environment the script starts its N ranks itself (torch.distributed.run on
+127.0.0.1); under torchrun it is one of the ranks.  Prints ONE JSON line (rank 0).  Inputs are seeded synthetic forests (workloads.py).  `value` is nodes/s
 with inputs resident in HBM; `e2e` is the same step through the host-buffer entry point with the copies
 inside the timed region.  At N > 1 every rank runs its own forest of the same shape (trees are
 independent: no collective on the data path) and the time is the max over ranks.
@@ -81,7 +82,47 @@ def time_oracle(w: wl.Workload, budget_s: float):
                 oracle_step(w, sub, x)
             dt = (time.perf_counter() - t0) / runs
     return (sub.n_nodes / dt,
-            f"first {sub.n_trees} of {w.forest.n_trees} trees ({sub.n_nodes} nodes), {runs} run(s), {dt:.2f} s each")
+            f"first {sub.n_trees} of {w.forest.n_trees} trees ({sub.n_nodes} nodes), {runs} run(s), {dt:.2f} s each",
+            sub.n_trees)
+
+
+def _oracle_worker(task):
+    """One process of the parallel baseline: the checker, as it stands, over its share of the trees (one thread)."""
+    child_ptr, child_idx, x, W, U, b, n_nodes = task
+    from threadpoolctl import threadpool_limits
+    from oracle import schedule as osched
+    from oracle import treelstm as ot
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        osched.schedule(child_ptr, child_idx, n_nodes)
+        ot.forward(child_ptr, child_idx, x, W, U, b)
+        return n_nodes, time.perf_counter() - t0
+
+
+def time_oracle_parallel(w: wl.Workload, trees_per_worker: int, max_workers: int = 32):
+    """nodes/s of the checker with the trees dealt out over worker processes (trees are independent units).
+    Workers are started with `spawn`: the parent process already holds a CUDA context."""
+    import multiprocessing as mp
+    try:
+        avail = len(os.sched_getaffinity(0))
+    except AttributeError:  # pragma: no cover
+        avail = os.cpu_count() or 1
+    cores = max(1, min(avail, max_workers, w.forest.n_trees // max(trees_per_worker, 1) or 1))
+    tasks = []
+    for k in range(cores):
+        trees = np.arange(k * trees_per_worker, min((k + 1) * trees_per_worker, w.forest.n_trees))
+        sub, nodes = wl.subforest(w.forest, trees)
+        tasks.append((sub.child_ptr, sub.child_idx, w.x_rows(nodes), w.W, w.U, w.b, sub.n_nodes))
+    one, one_nodes = wl.subforest(w.forest, np.arange(1))
+    warm = (one.child_ptr, one.child_idx, w.x_rows(one_nodes), w.W, w.U, w.b, one.n_nodes)
+    ctx = mp.get_context("spawn")
+    with ctx.Pool(cores) as pool:
+        pool.map(_oracle_worker, [warm] * cores, chunksize=1)  # untimed: process start-up and imports
+        t0 = time.perf_counter()
+        done = pool.map(_oracle_worker, tasks, chunksize=1)
+        dt = time.perf_counter() - t0
+    nodes = sum(d[0] for d in done)
+    return nodes / dt, cores, f"{cores} processes x {trees_per_worker} trees ({nodes} nodes), {dt:.2f} s"
 
 
 def run_reference(args):
@@ -171,7 +212,8 @@ class ClockSampler:
 
 
 def algorithmic_work(w: wl.Workload, n_leaves: int):
-    """Minimal flops and bytes of one forward (what the method must compute and touch)."""
+    """Minimal flops and bytes of one forward (what the method must compute and touch): every row once, the weights
+    once at their own type, nothing round-tripped."""
     f = w.forest
     N, E, D, H = f.n_nodes, f.n_edges, w.D, w.H
     n_int = N - n_leaves
@@ -182,31 +224,42 @@ def algorithmic_work(w: wl.Workload, n_leaves: int):
     return flops, bytes_
 
 
-def level_kernel_bytes(w: wl.Workload, n_leaves: int):
-    """Algorithmic bytes of the level loop alone: P rows in, child h/c rows in, h/c rows out, U once."""
+def level_loop_bytes(w: wl.Workload, n_leaves: int):
+    """(algorithmic, design) bytes of the level loop alone.  Algorithmic: h and c rows of the internal nodes out, h and c
+    rows of every child in, the recurrent weights once at their own type, the index arrays.  Design: what the kernels
+    add on top of that by construction (the fp32 input-projection rows of the internal nodes they read back; the
+    bf16 copies of h the tensor-core paths keep)."""
     f = w.forest
     n_int = f.n_nodes - n_leaves
     H = w.H
-    return n_int * (4 * H * 4 + 2 * H * 4) + f.n_edges * 2 * H * 4 + 4 * H * H * 4 + 4 * (2 * n_int + f.n_edges)
+    ws = 2 if w.precision == "bf16" else 4
+    algorithmic = n_int * 2 * H * 4 + f.n_edges * 2 * H * 4 + 4 * H * H * ws + 4 * (2 * n_int + f.n_edges)
+    design = n_int * 4 * H * 4
+    if w.precision == "bf16":
+        design += (n_int + f.n_edges) * H * 2
+    return algorithmic, design
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of the named kernel on the named workload
-# (one full-metric capture each, summarised under profiles/); None where the kernel has changed since its counters were taken.
+# ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch (of all launches of one step, for the per-level loop)
+# of the named kernels on the named workload, from the captures summarised under profiles/; None where a kernel has
+# changed since its counters were taken.
 MEASURED_TRAFFIC = {
-    ("small_levels_kernel", 2): 5647616 + 0,            # whole workload captured
-    ("small_levels_kernel", 4): 625942528 + 269811968,  # whole workload captured
-    ("small_levels_f32_kernel", 1): 2225152 + 256,      # whole workload captured
-    # captured on 8192 of the 65536 trees (194583 nodes: 408579072 + 2036310000 bytes) and scaled by the node count:
-    # every row is read and written once, so traffic grows in proportion
-    ("gemm_tc_kernel<EPI_XPROJ>", 5): int((408579072 + 2036310000) * (1571637 / 194583)),
+    ("small_levels_kernel", 2): None,
+    ("small_levels_kernel", 4): None,
+    ("small_levels_f32_kernel", 1): None,
+    ("gemm_tc_kernel<EPI_XPROJ>", 5): None,
+    ("per-level loop", 3): None,
+    ("per-level loop", 5): None,
 }
 
 
 def roofline_of(job, phases, t_step_s, pk):
-    """Roofline object of the dominant kernel of one step, and the whole step against its binding bound.
+    """Roofline object of the dominant kernel of one step, the same for both phases, and the whole step against its
+    binding bound.
 
-    phases: per step (input projection ms, level loop ms, batching analysis ms) from CUDA events recorded by the library on the
-    launching stream around those kernels.
+    phases: per step (input projection ms, level loop ms, batching analysis ms) from CUDA events recorded by the
+    library on the launching stream around those kernels.  The tensor peak is the burst figure of the measured
+    bf16 GEMM (the higher of the two measured ones) for every workload.
     """
     w = job.w
     f = w.forest
@@ -215,37 +268,49 @@ def roofline_of(job, phases, t_step_s, pk):
     xproj_ms = statistics.mean(p[0] for p in phases)
     lvl_ms = statistics.mean(p[1] for p in phases)
     flops, bytes_ = algorithmic_work(w, job.n_leaves)
-    tensor_peak = pk["bf16_tflops"] if t_step_s < 0.05 else pk["bf16_tflops_sustained"]
-    t_tensor = flops / (tensor_peak * 1e12)
+    tensor_peak = pk["bf16_tflops"]
+    t_tensor = flops / (tensor_peak * 1e12) if w.precision == "bf16" else 0.0
     t_hbm = bytes_ / (pk["hbm_gbs"] * 1e9)
     path_frac = max(t_tensor, t_hbm) / t_step_s
-    if w.precision == "bf16" and xproj_ms >= lvl_ms:
-        # input projection GEMM: algorithmic flops = three gate blocks for leaves, four for internal nodes
-        xflops = (job.n_leaves * 6 + n_int * 8) * D * H
-        achieved = xflops / (xproj_ms * 1e-3) / 1e12
-        kernel = "gemm_tc_kernel<EPI_XPROJ>"
-        roof = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
-                "frac": achieved / tensor_peak}
+
+    # input projection: algorithmic flops = three gate blocks for leaves, four for internal nodes
+    xflops = (job.n_leaves * 6 + n_int * 8) * D * H
+    x_ach = xflops / (xproj_ms * 1e-3) / 1e12 if xproj_ms > 0 else 0.0
+    lbytes, ldesign = level_loop_bytes(w, job.n_leaves)
+    l_ach = lbytes / (lvl_ms * 1e-3) / 1e9 if lvl_ms > 0 else 0.0
+    lflops = n_int * 6 * H * H + E * 2 * H * H
+    if w.precision != "bf16":
+        lkernel = "small_levels_f32_kernel" if w.H <= 192 else "persistent_kernel / level_kernel (fp32 ALUs)"
+    elif job.small:
+        lkernel = "small_levels_kernel"
     else:
-        lbytes = level_kernel_bytes(w, job.n_leaves)
-        achieved = lbytes / (lvl_ms * 1e-3) / 1e9
-        if w.precision != "bf16":
-            kernel = "small_levels_f32_kernel" if w.H <= 192 else "persistent_kernel / level_kernel (fp32 ALUs)"
-        elif job.small and job.n_wide > 0:
-            kernel = f"level loop: {job.n_wide} wide levels as per-level launches, then small_levels_kernel"
-        elif job.small:
-            kernel = "small_levels_kernel"
-        else:
-            kernel = "level loop: gather_kernel + gemm_tc_kernel<EPI_LEVEL> + gemm_tc_kernel<EPI_G> per level"
-        roof = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / pk["hbm_gbs"]}
-    roof["traffic"] = MEASURED_TRAFFIC.get((roof["kernel"], w.index))
+        lkernel = "per-level loop"
+    phases_out = {
+        "input_projection": {"kernel": "gemm_tc_kernel<EPI_XPROJ>" if w.precision == "bf16" else "xproj_simt_kernel",
+                             "ms": xproj_ms, "flops": xflops, "tflops": x_ach,
+                             "frac_of_tensor_peak": x_ach / tensor_peak if w.precision == "bf16" else None},
+        "level_loop": {"kernel": lkernel, "ms": lvl_ms, "algorithmic_bytes": lbytes, "design_bytes": ldesign,
+                       "gbs": l_ach, "frac_of_hbm_peak": l_ach / pk["hbm_gbs"], "flops": lflops,
+                       "tflops": lflops / (lvl_ms * 1e-3) / 1e12 if lvl_ms > 0 else 0.0},
+        "schedule_ms": statistics.mean(p[2] for p in phases),
+    }
+    if w.precision == "bf16" and xproj_ms >= lvl_ms:
+        kernel = "gemm_tc_kernel<EPI_XPROJ>"
+        roof = {"bound": "tensor", "kernel": kernel, "achieved": x_ach, "peak": tensor_peak, "unit": "TFLOP/s",
+                "frac": x_ach / tensor_peak, "frac_of_sustained_peak": x_ach / pk["bf16_tflops_sustained"]}
+    else:
+        kernel = lkernel
+        roof = {"bound": "hbm", "kernel": kernel, "achieved": l_ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": l_ach / pk["hbm_gbs"], "algorithmic_bytes": lbytes, "design_bytes": ldesign}
+        if kernel == "per-level loop":
+            roof["kernel"] = "per-level loop: childsum_kernel + gemm_tc_kernel<EPI_F> + gemm_tc_kernel<EPI_LEVEL> per level"
+    roof["traffic"] = MEASURED_TRAFFIC.get((kernel, w.index))
     roof["peak_source"] = pk["source"]
     roof["ms_per_launch"] = xproj_ms if roof["bound"] == "tensor" else lvl_ms
     roof["xproj_ms"] = xproj_ms
     roof["levels_ms"] = lvl_ms
-    roof["schedule_ms"] = statistics.mean(p[2] for p in phases)   # batching analysis alone (start of step to start of forward)
-    return roof, path_frac
+    roof["schedule_ms"] = phases_out["schedule_ms"]   # batching analysis alone (start of step to start of forward)
+    return roof, path_frac, phases_out
 
 
 class GpuJob:
@@ -273,16 +338,18 @@ class GpuJob:
         self.c = torch.empty((f.n_nodes, self.ldh), dtype=torch.float32, device=device)
         jdb.jdb_schedule(self.forest, self.sched, self.sws)
         self.n_levels, self.n_leaves = self.sched.n_levels, self.sched.n_leaves
+        self.level_sizes = np.diff(self.sched.level_ptr[:self.n_levels + 1].cpu().numpy()).tolist()
         self.small = self.precision == jdb.BF16 and w.H <= 192 and mode != jdb.MODE_PER_LEVEL
-        self.sched.n_leaves = -1  # size the workspace for a schedule whose counts stay on the device
+        # the cooperative level loops read the level count on the device, so the analysis need not synchronise
+        # and the forward can defer its status to one check after the timed loop; per-level launches need the
+        # counts on the host, so there the analysis synchronises inside the step
+        self.async_schedule = self.small or self.precision == jdb.FP32
+        if self.async_schedule:
+            self.sched.n_leaves = -1  # size the workspace for a schedule whose counts stay on the device
         self.fws = jdb.forward_workspace(self.forest, self.sched, w.D, w.H, self.precision)
         self.events = None
-        # the cooperative level loop reads the level count on the device, so the analysis need not synchronise
-        # and the forward can defer its status to one check after the timed loop
-        # ... unless the forest has levels wide enough for launches of their own: the host then needs the counts
-        self.n_wide = self.sched.n_wide_levels if (self.small and mode == jdb.MODE_AUTO) else 0
         self.plan = jdb.StepPlan(self.forest, self.sched, self.sws, self.x, self.packed, w.D, w.H, self.precision,
-                                 self.h, self.c, self.fws, mode=mode, async_schedule=self.small and self.n_wide == 0)
+                                 self.h, self.c, self.fws, mode=mode, async_schedule=self.async_schedule)
 
     def step(self):
         self.plan.set_events(self.events)
@@ -297,10 +364,8 @@ class GpuJob:
             persistent = self.mode == jdb.MODE_PERSISTENT or (self.mode == jdb.MODE_AUTO and (self.w.H <= 192 or self.n_levels > 6))
             return sched + 1 + (1 if persistent else levels)
         if self.small:
-            own = min(self.n_wide, levels)           # leading wide levels: leaf G GEMM + 3 launches each, no G after the last
-            coop = 1 if levels > own else 0
-            return sched + 2 + (3 * own if own else 0) + coop   # level-order copy, projection GEMM, level loop
-        return sched + 2 + 3 * levels                # + leaf G GEMM and 3 per level, no G after the last
+            return sched + 2 + (1 if levels else 0)   # level-order copy, projection GEMM, cooperative level loop
+        return sched + 2 + 3 + 3 * levels             # + three layout kernels, and child sums + two GEMMs per level
 
 
 def time_steps(job: GpuJob, steps: int, warmup: int, flush, timed_events=False):
@@ -328,6 +393,36 @@ def time_steps(job: GpuJob, steps: int, warmup: int, flush, timed_events=False):
     return total, level_ms
 
 
+def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device):
+    """The same step through the host-buffer entry point: pinned host arrays in, pinned host arrays out, the
+    copies inside the timed region.  Returns (per-step ms, h2d bytes, d2h bytes)."""
+    torch, jdb = job.torch, job.jdb
+    f = w.forest
+    dt = torch.bfloat16 if job.precision == jdb.BF16 else torch.float32
+    hx = torch.from_numpy(w.x_full()).to(dt).pin_memory()
+    hcp, hci = torch.from_numpy(f.child_ptr).pin_memory(), torch.from_numpy(f.child_idx).pin_memory()
+    hh = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
+    hc = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
+    x_dtype = jdb.BF16 if dt == torch.bfloat16 else jdb.FP32
+    hws = jdb.forward_host_workspace(f.n_nodes, f.n_edges, w.D, w.H, job.precision, x_dtype, device)
+    for _ in range(max(warmup, 3)):
+        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(steps):
+        flush.add_(1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
+        e1.record()
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    h2d = hcp.numel() * 4 + hci.numel() * 4 + hx.numel() * hx.element_size()
+    d2h = hh.numel() * 4 + hc.numel() * 4
+    return ms, h2d, d2h
+
+
 def rank_workload(config: int, rank: int, n_trees=None) -> wl.Workload:
     """Every rank draws its own forest of the workload's shape (weak scaling over independent trees)."""
     return wl.make_workload(config, n_trees=n_trees, seed=None if rank == 0 else wl.BASE_SEED + config + 1000 * rank)
@@ -347,6 +442,14 @@ def job_totals(seconds: float, nodes: int, world: int, device):
     return float(t.item()), float(n.item())
 
 
+def config_entry(idx, w, job, times, steps, value, roofline, path_frac, phases):
+    f = w.forest
+    return {"config": idx, "workload": w.name, "nodes": f.n_nodes, "edges": f.n_edges, "levels": job.n_levels,
+            "level_sizes": job.level_sizes, "batching_ratio": f.n_nodes / max(job.n_levels, 1), "steps": steps,
+            "ms_per_step": sum(times) / len(times), "ms_median": statistics.median(times), "ms_min": min(times),
+            "value": value, "roofline": roofline, "path_frac_of_roofline": path_frac, "phases": phases}
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -355,8 +458,21 @@ def run_gpu(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.rendezvous_only:
+        # a check of the launcher that needs no GPU: the ranks meet over gloo, reduce the totals, rank 0 prints
+        dist.init_process_group("gloo")
+        w = rank_workload(1, rank)
+        t_s, total_nodes = job_totals(1.0 + rank, w.forest.n_nodes, world, torch.device("cpu"))
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "n_gpus": world, "rendezvous_only": True, "max_seconds": t_s,
+                              "total_nodes": total_nodes}))
+        dist.barrier()
+        dist.destroy_process_group()
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank} has no GPU: {torch.cuda.device_count()} visible, {world} ranks")
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
@@ -366,6 +482,7 @@ def run_gpu(args):
     pk = peaks()
     mode = {"auto": jdb.MODE_AUTO, "level": jdb.MODE_PER_LEVEL, "persistent": jdb.MODE_PERSISTENT}[args.mode]
     w = rank_workload(args.config, rank, args.trees)
+    f = w.forest
     job = GpuJob(w, device, mode)
     flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=device)
 
@@ -382,63 +499,42 @@ def run_gpu(args):
     times, phases = time_steps(job, args.steps, 0, flush, timed_events=True)
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    t_s, total_nodes = job_totals(sum(times) / 1e3, w.forest.n_nodes, world, device)
+    t_s, total_nodes = job_totals(sum(times) / 1e3, f.n_nodes, world, device)
     value = total_nodes * args.steps / t_s
-
-    # end to end from pinned host buffers through the host entry point
-    f = w.forest
-    dt = torch.bfloat16 if job.precision == jdb.BF16 else torch.float32
-    hx = torch.from_numpy(w.x_full()).to(dt).pin_memory()
-    hcp, hci = torch.from_numpy(f.child_ptr).pin_memory(), torch.from_numpy(f.child_idx).pin_memory()
-    hh = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
-    hc = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
-    x_dtype = jdb.BF16 if dt == torch.bfloat16 else jdb.FP32
-    hws = jdb.forward_host_workspace(f.n_nodes, f.n_edges, w.D, w.H, job.precision, x_dtype, device)
-    for _ in range(max(args.warmup, 3)):
-        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
-    torch.cuda.synchronize()
-    e2e_ms = []
-    for _ in range(args.steps):
-        flush.add_(1)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
-        e1.record()
-        e1.synchronize()
-        e2e_ms.append(e0.elapsed_time(e1))
-    t_e2e_s, _ = job_totals(sum(e2e_ms) / 1e3, w.forest.n_nodes, world, device)
-    e2e_value = total_nodes * args.steps / t_e2e_s
-    h2d = hcp.numel() * 4 + hci.numel() * 4 + hx.numel() * hx.element_size()
-    d2h = hh.numel() * 4 + hc.numel() * 4
+    roofline, path_frac, phases_out = roofline_of(job, phases, t_s / args.steps, pk)
+    main_entry = config_entry(args.config, w, job, times, args.steps, value, roofline, path_frac, phases_out)
     n_levels_main, launches_main = job.n_levels, job.launches_per_step()
+    precision_main, packed_main = job.precision, job.packed
+
+    # end to end from pinned host buffers through the host entry point (the resident buffers are released first)
+    job.plan = None
+    job.x = job.h = job.c = job.fws = job.sws = None
+    torch.cuda.empty_cache()
+    e2e_ms, h2d, d2h = time_e2e(w, job, args.steps, args.warmup, flush, device)
+    t_e2e_s, _ = job_totals(sum(e2e_ms) / 1e3, f.n_nodes, world, device)
+    e2e_value = total_nodes * args.steps / t_e2e_s
+    del job
+    torch.cuda.empty_cache()
 
     if rank == 0:
-        roofline, path_frac = roofline_of(job, phases, t_s / args.steps, pk)
         per_config = []
         if args.all_configs and world == 1:
-            del job, hws
-            torch.cuda.empty_cache()
             for idx in (1, 2, 3, 4, 5):
                 if idx == args.config:
-                    per_config.append({"config": idx, "workload": w.name, "nodes": f.n_nodes, "levels": n_levels_main,
-                                       "batching_ratio": f.n_nodes / max(n_levels_main, 1),
-                                       "ms_per_step": 1e3 * t_s / args.steps, "ms_median": statistics.median(times),
-                                       "ms_min": min(times), "value": value, "roofline": roofline,
-                                       "path_frac_of_roofline": path_frac})
+                    per_config.append(main_entry)
                     continue
                 wi = wl.make_workload(idx)
                 ji = GpuJob(wi, device, mode)
-                k = 5 if idx == 5 else 10
-                ti, ph = time_steps(ji, k, 3, flush, timed_events=True)
-                ri, pf = roofline_of(ji, ph, sum(ti) / 1e3 / k, pk)
-                per_config.append({"config": idx, "workload": wi.name, "nodes": wi.forest.n_nodes, "levels": ji.n_levels,
-                                   "batching_ratio": wi.forest.n_nodes / max(ji.n_levels, 1),
-                                   "ms_per_step": sum(ti) / k, "ms_median": statistics.median(ti), "ms_min": min(ti), "value": wi.forest.n_nodes * k / (sum(ti) / 1e3),
-                                   "roofline": ri, "path_frac_of_roofline": pf})
+                ti, ph = time_steps(ji, args.steps, args.warmup, flush, timed_events=True)
+                ri, pf, po = roofline_of(ji, ph, sum(ti) / 1e3 / args.steps, pk)
+                per_config.append(config_entry(idx, wi, ji, ti, args.steps, wi.forest.n_nodes * args.steps / (sum(ti) / 1e3), ri, pf, po))
                 del ji, wi
                 torch.cuda.empty_cache()
-        cpu_v, cpu_sample = time_oracle(w, args.cpu_budget)
+        cpu_v, cpu_sample, cpu_trees = time_oracle(w, args.cpu_budget)
+        cpu_par = None
+        if args.cpu_budget >= 1.0:
+            pv, pcores, psample = time_oracle_parallel(w, max(1, cpu_trees))
+            cpu_par = {"value": pv, "unit": UNIT, "cores": pcores, "kind": "oracle", "sample": psample}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * t_s / args.steps, "ms_median": statistics.median(times), "ms_min": min(times),
@@ -455,8 +551,10 @@ def run_gpu(args):
             "gpu_launches": launches_main * args.steps,
             "roofline": roofline,
             "path_frac_of_roofline": path_frac,
+            "phases": phases_out,
             "batching_ratio": f.n_nodes / max(n_levels_main, 1),   # cells evaluated per batched step: Section 3's batching ratio at cell granularity
-            "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample},
+            "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample,
+                             "parallel_over_trees": cpu_par},
             "per_config": per_config,
         }
         print(json.dumps(line))
@@ -465,23 +563,42 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def launcher_command(n_ranks: int, argv, port: int):
+    """The command that starts this script as `n_ranks` ranks of one node (what a driver would type itself)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="jdb", choices=["jdb", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5],
+                    help="workload of the top-level figures (default: the largest one, 5); the others go under per_config")
     ap.add_argument("--trees", type=int, default=None,
                     help="shrink the forest to this many trees of the same shape (profiler captures; not a bench value)")
     ap.add_argument("--mode", default="auto", choices=["auto", "level", "persistent"])
-    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of CPU time for the cpu_baseline sample")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of CPU time for each cpu_baseline sample")
     ap.add_argument("--all-configs", dest="all_configs", action="store_true", default=True,
                     help="also time the other four workloads and list them under per_config (1 GPU only)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
+    ap.add_argument("--rendezvous-only", action="store_true",
+                    help="start the ranks, reduce the totals over gloo on the CPU and print them: checks the launcher, times nothing")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started bare: become the launcher of the N ranks (rank 0 prints the line)
+        raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:], free_port())))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -35,7 +35,9 @@ typedef enum {
     JDB_ERR_WORKSPACE = 3,     /* workspace or packed-weight buffer too small                    */
     JDB_ERR_UNSUPPORTED = 4,   /* sizes outside what the kernels were built for                  */
     JDB_ERR_CUDA = 5,          /* a CUDA runtime call failed (see jdb_last_cuda_error)           */
-    JDB_ERR_TIMEOUT = 6        /* a bounded device-side wait ran out; outputs are undefined      */
+    JDB_ERR_TIMEOUT = 6,       /* a bounded device-side wait ran out; outputs are undefined      */
+    JDB_ERR_CHECK = 7          /* JDB_FLAG_DEBUG_CHECKS: a kernel met an index outside its arrays (the access was
+                                  skipped; see jdb_debug_report)                                  */
 } jdb_status;
 
 /* precision of the GEMM operands; accumulation and the c/h state are always fp32 */
@@ -44,7 +46,27 @@ enum { JDB_FP32 = 0, JDB_BF16 = 1 };
 enum { JDB_MODE_AUTO = 0, JDB_MODE_PER_LEVEL = 1, JDB_MODE_PERSISTENT = 2 };
 
 /* jdb_opts.flags */
-enum { JDB_FLAG_NO_SYNC = 1 }; /* jdb_treelstm_forward never synchronises; ask jdb_sched_status afterwards */
+enum {
+    JDB_FLAG_NO_SYNC = 1,      /* jdb_treelstm_forward never synchronises; ask jdb_sched_status afterwards */
+    JDB_FLAG_DEBUG_CHECKS = 2  /* every kernel of the forward pass checks the indices it is about to follow (child ids,
+                                  positions in level order, level offsets, rows of the workspace arrays) against the
+                                  sizes of the arrays they index, skips an access that would leave them and records the
+                                  first offender in sched->meta; the call then synchronises and returns JDB_ERR_CHECK.
+                                  Slower; meant for tests and for bringing up a new caller.                          */
+};
+
+/* jdb_opts.tuning: 0 takes the library's defaults (the measured best, which the environment variables JDB_GEMM_PAIR,
+ * JDB_GEMM_ISSUERS, JDB_PDL and JDB_P_TMA may change, read at every call).  With JDB_TUNE_SET the other bits
+ * replace those defaults for this call; every combination computes the same values. */
+enum {
+    JDB_TUNE_SET = 1,
+    JDB_TUNE_PAIR_XPROJ = 2,    /* input-projection GEMM as CTA pairs (forests of at least 256 rows per SM)          */
+    JDB_TUNE_PAIR_LEVEL = 4,    /* per-level gate GEMM as CTA pairs                                                  */
+    JDB_TUNE_PAIR_FORGET = 8,   /* per-level forget-gate GEMM as CTA pairs (launches with at least 32 tiles per pair)*/
+    JDB_TUNE_TWO_ISSUERS = 16,  /* two MMA-issuing warps per lone CTA, half of the tile's columns each               */
+    JDB_TUNE_NO_PDL = 32,       /* ordinary launches instead of programmatic dependent launches                      */
+    JDB_TUNE_PLAIN_STORES = 64  /* level-ordered outputs through the load/store units instead of TMA stores           */
+};
 
 #define JDB_META_INTS 16 /* size of jdb_sched.meta in int32 */
 
@@ -58,8 +80,8 @@ typedef struct {
     int32_t n_edges;
 } jdb_forest;
 
-/* The depth table of Section 4.2.  depth(v) = 0 for a leaf, else 1 + max over its children, so that
- * "nodes at the same depth are independent of each other" and levels run in ascending order.
+/* The depth table of Section 4.2.  depth(v) = 0 for a leaf, else 1 + max over its children: no node depends on
+ * another node of its own depth, and levels run in ascending order.
  * All arrays are caller-allocated device memory. */
 typedef struct {
     int32_t *depth;     /* [n_nodes]                                                            */
@@ -70,8 +92,8 @@ typedef struct {
     int32_t n_levels;   /* host; written by jdb_schedule, -1 after jdb_schedule_async            */
     int32_t n_leaves;   /* host; = level_ptr[1]; -1 after jdb_schedule_async                     */
     int32_t n_wide_levels; /* host; how many of the levels 1, 2, ... in a row hold at least 65536 nodes
-                           (such a level fills the GPU with launches of its own; the forward pass starts
-                           its single-launch level loop after them); -1 after jdb_schedule_async    */
+                           (a statistic of the depth table; the forward pass does not depend on it);
+                           -1 after jdb_schedule_async                                             */
     int32_t reserved0;  /* 0 */
 } jdb_sched;
 
@@ -79,7 +101,7 @@ typedef struct {
     int32_t precision;  /* JDB_FP32 | JDB_BF16: must match the packed weights                    */
     int32_t mode;       /* JDB_MODE_*                                                            */
     int32_t flags;      /* JDB_FLAG_* ORed together                                              */
-    int32_t reserved1;
+    int32_t tuning;     /* JDB_TUNE_* ORed together; 0 = defaults                                */
     uint64_t barrier_timeout_ns; /* limit of one grid-barrier wait in persistent mode; 0 = 2 s   */
     /* Optional timing hooks: cudaEvent_t handles (as void*, NULL = none) recorded on `stream` before
      * the input projection, after it, and after the level loop, so that a caller can time the two
@@ -157,7 +179,10 @@ size_t jdb_forward_workspace_bytes(int32_t n_nodes, int32_t n_internal_bound, in
  * Asynchronous on `stream` unless the level loop runs as one cooperative launch (persistent mode, or a
  * schedule from jdb_schedule_async), in which case the call synchronises at the end to report
  * JDB_ERR_NOT_A_FOREST / JDB_ERR_TIMEOUT.  With JDB_FLAG_NO_SYNC it does not synchronise either (as long as
- * the level count is known or H <= 192) and those two conditions are reported by jdb_sched_status. */
+ * the level count is known or H <= 192) and those two conditions are reported by jdb_sched_status.
+ * A bounded wait that runs out inside one of the per-level launches (which are asynchronous) is likewise
+ * visible through jdb_sched_status only.  JDB_BF16 with H > 192 runs one set of launches per level and needs the
+ * level count on the host: after jdb_schedule_async the call first synchronises once to read it. */
 jdb_status jdb_treelstm_forward(const jdb_forest *forest, const jdb_sched *sched, const void *x,
                                 int32_t x_dtype, int64_t ldx, const void *packed, int32_t D, int32_t H,
                                 float *h, float *c, int64_t ldh, const jdb_opts *opts, void *ws,
@@ -169,6 +194,13 @@ jdb_status jdb_treelstm_forward(const jdb_forest *forest, const jdb_sched *sched
  * JDB_FLAG_NO_SYNC (deferred error reporting of the depth-ordered execution of Section 4.2). */
 jdb_status jdb_sched_status(const jdb_sched *sched, int32_t *n_levels_out, int32_t *n_leaves_out, void *stream);
 
+/* What JDB_FLAG_DEBUG_CHECKS recorded for the calls enqueued so far on this schedule (synchronises `stream`):
+ * out[0] which check failed first (0 none; 1 node id from perm, 2 child id, 3 position in level order, 4 edge slot,
+ * 5 parent row, 6 level offset, 7 edge offset), out[1] the offending value, out[2] the bound it was held against
+ * (valid values are 0 .. bound-1), out[3] the position, slot, node or level at which it was met.  `out` is a host array.
+ * The companion of the depth-ordered execution of Section 4.2 for callers that assemble schedules themselves. */
+jdb_status jdb_debug_report(const jdb_sched *sched, int32_t out[4], void *stream);
+
 /* ---- one call from host buffers (what a user without device arrays calls) -------------------- */
 
 /* Device scratch needed by jdb_treelstm_forward_host (CSR, x, schedule, h, c and both workspaces). */
@@ -177,9 +209,10 @@ size_t jdb_forward_host_workspace_bytes(int32_t n_nodes, int32_t n_edges, int32_
 
 /* child_ptr, child_idx, x, h, c are HOST pointers (pinned memory makes the copies asynchronous);
  * x is dense [n_nodes, D], h and c dense [n_nodes, H].  Copies the inputs to `dev_ws`, runs the
- * analysis and the forward there, copies h and c back and synchronises the stream ONCE, at the end;
- * JDB_ERR_NOT_A_FOREST and JDB_ERR_TIMEOUT are reported then.  n_levels_out (host, may be NULL)
- * receives the level count. */
+ * analysis and the forward there, copies h and c back and synchronises the stream at the end, where
+ * JDB_ERR_NOT_A_FOREST and JDB_ERR_TIMEOUT are reported.  That is the only synchronisation for JDB_FP32 and for
+ * JDB_BF16 with H <= 192; JDB_BF16 with H > 192 launches per level and synchronises once more, after the analysis,
+ * to read the level count.  n_levels_out (host, may be NULL) receives the level count. */
 jdb_status jdb_treelstm_forward_host(const int32_t *child_ptr, const int32_t *child_idx, int32_t n_nodes,
                                      int32_t n_edges, const void *x, int32_t x_dtype, const void *packed,
                                      int32_t D, int32_t H, float *h, float *c, const jdb_opts *opts,

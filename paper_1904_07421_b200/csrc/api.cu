@@ -32,6 +32,14 @@ jdb_status read_meta(const int32_t* meta_dev, int32_t* meta_host, cudaStream_t s
     return JDB_OK;
 }
 
+// what the device recorded about the calls enqueued so far
+jdb_status meta_status(const int32_t* meta) {
+    if (meta[META_ERROR] != 0 || meta[META_UNFINISHED] != 0) return JDB_ERR_NOT_A_FOREST;
+    if (meta[META_TIMEOUT] != 0) return JDB_ERR_TIMEOUT;
+    if (meta[META_CHECK] != 0) return JDB_ERR_CHECK;
+    return JDB_OK;
+}
+
 jdb_status check_forest_args(const jdb_forest* f) {
     if (!f || f->n_nodes < 0 || f->n_edges < 0) return JDB_ERR_INVALID_ARG;
     if (f->n_nodes > 0 && !f->child_ptr) return JDB_ERR_INVALID_ARG;
@@ -80,6 +88,7 @@ const char* jdb_status_string(jdb_status s) {
         case JDB_ERR_UNSUPPORTED: return "size not supported by the compiled kernels";
         case JDB_ERR_CUDA: return "CUDA runtime error";
         case JDB_ERR_TIMEOUT: return "device-side wait timed out";
+        case JDB_ERR_CHECK: return "debug checks: a kernel met an index outside its array (access skipped; see jdb_debug_report)";
     }
     return "unknown status";
 }
@@ -201,25 +210,33 @@ jdb_status jdb_treelstm_forward(const jdb_forest* forest, const jdb_sched* sched
     a.ev_levels_done = (cudaEvent_t)opts->ev_levels_done;
     a.trace = (unsigned long long*)opts->trace;
     a.trace_cap = opts->trace ? opts->trace_cap : 0;
+    a.tuning = opts->tuning;
+    a.debug = (opts->flags & JDB_FLAG_DEBUG_CHECKS) ? 1 : 0;
 
-    if (mode == JDB_MODE_PERSISTENT)
-        JDB_CUDA_TRY(cudaMemsetAsync(sched->meta + META_TIMEOUT, 0, 2 * sizeof(int32_t), st));
+    // what an earlier forward on this schedule may have left: the timeout word, the barrier counter, the debug record
+    JDB_CUDA_TRY(cudaMemsetAsync(sched->meta + META_TIMEOUT, 0, 2 * sizeof(int32_t), st));
+    if (a.debug) JDB_CUDA_TRY(cudaMemsetAsync(sched->meta + META_CHECK, 0, 4 * sizeof(int32_t), st));
     const uint64_t tmo = opts->barrier_timeout_ns ? opts->barrier_timeout_ns : 2000000000ull;
-    // AUTO with the level sizes known on the host: levels wide enough to fill the GPU by themselves run as their
-    // own launches, the cooperative loop takes over at the first narrower one
-    const int n_wide = (tc_small && known && opts->mode == JDB_MODE_AUTO && sched->n_wide_levels > 0) ? sched->n_wide_levels : 0;
     if (tc)
-        s = forward_tc_enqueue(a, pk + L.total, n_levels_host, n_internal_bound, ws, tc_small, n_wide, tmo, st);
+        s = forward_tc_enqueue(a, pk + L.total, n_levels_host, n_internal_bound, ws, tc_small, tmo, st);
     else
         s = forward_enqueue(a, n_levels_host, n_internal_bound, mode, tmo, st);
     if (s != JDB_OK) return s;
-    if (mode == JDB_MODE_PERSISTENT && !(opts->flags & JDB_FLAG_NO_SYNC)) {
+    if (a.debug || (mode == JDB_MODE_PERSISTENT && !(opts->flags & JDB_FLAG_NO_SYNC))) {
         int32_t meta[JDB_META_INTS];
         s = read_meta(sched->meta, meta, st);
         if (s != JDB_OK) return s;
-        if (meta[META_ERROR] != 0 || meta[META_UNFINISHED] != 0) return JDB_ERR_NOT_A_FOREST;
-        if (meta[META_TIMEOUT] != 0) return JDB_ERR_TIMEOUT;
+        return meta_status(meta);
     }
+    return JDB_OK;
+}
+
+jdb_status jdb_debug_report(const jdb_sched* sched, int32_t out[4], void* stream) {
+    if (!sched || !sched->meta || !out) return JDB_ERR_INVALID_ARG;
+    int32_t meta[JDB_META_INTS];
+    jdb_status s = read_meta(sched->meta, meta, (cudaStream_t)stream);
+    if (s != JDB_OK) return s;
+    for (int i = 0; i < 4; ++i) out[i] = meta[META_CHECK + i];
     return JDB_OK;
 }
 
@@ -230,9 +247,7 @@ jdb_status jdb_sched_status(const jdb_sched* sched, int32_t* n_levels_out, int32
     if (s != JDB_OK) return s;
     if (n_levels_out) *n_levels_out = meta[META_N_LEVELS];
     if (n_leaves_out) *n_leaves_out = meta[META_N_LEAVES];
-    if (meta[META_ERROR] != 0 || meta[META_UNFINISHED] != 0) return JDB_ERR_NOT_A_FOREST;
-    if (meta[META_TIMEOUT] != 0) return JDB_ERR_TIMEOUT;
-    return JDB_OK;
+    return meta_status(meta);
 }
 
 size_t jdb_forward_host_workspace_bytes(int32_t n_nodes, int32_t n_edges, int32_t D, int32_t H, int32_t precision,
@@ -303,10 +318,8 @@ jdb_status jdb_treelstm_forward_host(const int32_t* child_ptr, const int32_t* ch
     int32_t meta[JDB_META_INTS];
     s = read_meta(sch.meta, meta, st);
     if (s != JDB_OK) return s;
-    if (meta[META_ERROR] != 0 || meta[META_UNFINISHED] != 0) return JDB_ERR_NOT_A_FOREST;
-    if (meta[META_TIMEOUT] != 0) return JDB_ERR_TIMEOUT;
     if (n_levels_out) *n_levels_out = meta[META_N_LEVELS];
-    return JDB_OK;
+    return meta_status(meta);
 }
 
 }  // extern "C"

@@ -20,6 +20,7 @@ enum {
     META_TIMEOUT = 5,    // set by a grid barrier that gave up
     META_BARRIER = 6,    // grid barrier arrival counter (persistent mode)
     META_WIDE_LEVELS = 7, // how many levels 1, 2, ... in a row hold at least WIDE_LEVEL_NODES nodes
+    META_CHECK = 8,       // JDB_FLAG_DEBUG_CHECKS: which check failed first (0 = none), then value, bound, where
 };
 // A level this large keeps every SM busy with its own launches (gather + two GEMMs); smaller ones are cheaper
 // inside the cooperative level loop, whose cost per level is one grid barrier.
@@ -97,6 +98,8 @@ struct ForwardArgs {
     cudaEvent_t ev_begin, ev_xproj_done, ev_levels_done;  // optional timing hooks (null = none)
     unsigned long long* trace;                             // optional level trace (null = none)
     long long trace_cap;
+    int32_t tuning;                                        // jdb_opts.tuning
+    int32_t debug;                                         // 1: JDB_FLAG_DEBUG_CHECKS
 };
 size_t forward_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D, int32_t H, int32_t precision);
 jdb_status forward_enqueue(const ForwardArgs& a, int n_levels_host, int n_internal_bound, int mode,
@@ -118,7 +121,7 @@ size_t forward_tc_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D,
 // use_small: run the level loop as the one cooperative launch of forward_small.cu (H <= 192; n_levels may be
 // unknown on the host) instead of per-level launches (n_levels must be known)
 jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int n_levels, int n_internal_bound,
-                              void* ws, bool use_small, int n_wide, uint64_t timeout_ns, cudaStream_t st);
+                              void* ws, bool use_small, uint64_t timeout_ns, cudaStream_t st);
 
 // ---- forward_small.cu -------------------------------------------------------------------------
 bool small_levels_supported(int32_t H);

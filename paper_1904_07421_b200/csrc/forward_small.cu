@@ -196,8 +196,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                     }
                     cp_async_wait_all();
                     fence_proxy_async();
-                    named_bar(BAR_MAIN, MAIN_THREADS);
-                    if (s_abort) { alive = false; break; }
+                    if (named_bar_any(BAR_MAIN, MAIN_THREADS, !good || s_abort != 0)) { alive = false; break; }  // one verdict for all warps
                     stamp(level, 2, first && et0 == 0);
                     // ---- tensor cores: one product for all four gate blocks ----
                     if (tid == 0) {
@@ -225,7 +224,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                             pu[i] = __ldg(prow + 2 * Hp);
                         }
                     }
-                    if (!mbar_wait_warp(smem_u32(&bar_mma), mma_phase, abort)) *abort = 1;
+                    const bool mma_done = mbar_wait_warp(smem_u32(&bar_mma), mma_phase, abort);
+                    if (!mma_done) *abort = 1;
                     mma_phase ^= 1u;
                     tc_fence_after();
                     stamp(level, 4, first && et0 == 0);
@@ -258,8 +258,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                         }
                     }
                     tc_fence_before();
-                    named_bar(BAR_MAIN, MAIN_THREADS);
-                    if (s_abort) { alive = false; break; }
+                    if (named_bar_any(BAR_MAIN, MAIN_THREADS, !mma_done || s_abort != 0)) { alive = false; break; }
                     stamp(level, 5, first && et0 == 0);
                     // ---- cell arithmetic: one thread per (row, hidden unit) ----
 #pragma unroll
@@ -298,8 +297,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
             }
             if (!alive) break;
             if (level + 1 < n_levels) {
-                main_grid_barrier(a.meta, (unsigned)(level - a.first_level + 1) * active_ctas, a.timeout_ns, abort, tid);
-                if (s_abort) alive = false;
+                if (!main_grid_barrier(a.meta, (unsigned)(level - a.first_level + 1) * active_ctas, a.timeout_ns, abort, tid)) alive = false;
             }
             stamp(level, 7, true);
         }

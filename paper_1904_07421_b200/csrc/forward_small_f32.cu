@@ -181,8 +181,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
                         else *reinterpret_cast<float4*>(cs + e * CS_LD + 4 * q) = load_row4(crow, j0 + 4 * q, H, a.vec_ok);
                     }
                     cp_async_wait_all();
-                    named_bar(BAR_MAIN, MAIN_THREADS);
-                    if (s_abort) { alive = false; break; }
+                    if (named_bar_any(BAR_MAIN, MAIN_THREADS, !good || s_abort != 0)) { alive = false; break; }  // one verdict for all warps
                     stamp(level, 2, first && et0 == 0);
                     // ---- products: 2 edges x 4 outputs per thread, K ascending ----
                     float acc[2][4];
@@ -257,8 +256,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
             }
             if (!alive) break;
             if (level + 1 < n_levels) {
-                main_grid_barrier(a.meta, (unsigned)level * active_ctas, a.timeout_ns, abort, tid);
-                if (s_abort) alive = false;
+                if (!main_grid_barrier(a.meta, (unsigned)level * active_ctas, a.timeout_ns, abort, tid)) alive = false;
             }
             stamp(level, 7, true);
         }

@@ -8,14 +8,17 @@
 //              (level_order_x_kernel lays x out that way in one pass).  Leaf tiles compute only the i, o, u blocks
 //              and finish in the epilogue (c = sig(z_i) tanh(z_u), h = sig(z_o) tanh(c)); tiles of internal
 //              nodes store their four pre-activations to P.
-//   EPI_G      G_k = U_f h_k for every node that may be somebody's child.  The forget gate of child k under
-//              parent j is sig(W_f x_j + b_f + U_f h_k): the U_f h_k term depends on the child alone, so it is
-//              computed once per node as a plain GEMM over a level instead of once per edge on gathered rows.
+//   EPI_F      the per-child forget gates of one level.  The bf16 copy of h is kept in CHILD ORDER: the row of a
+//              node sits at the slot of the edge that leads to it, edges numbered by (position of the parent in
+//              level order, index in the parent's child list).  The children of a level's nodes are therefore one
+//              contiguous range of rows, sorted by parent: the product U_f h_k over them is a plain GEMM with TMA
+//              operands, and its epilogue turns every row into f_jk c_k = sig(W_f x_j + b_f + U_f h_k) c_k and adds
+//              the rows of one parent up (a segmented sum over the accumulator rows), so that only
+//              S_j = sum_k f_jk c_k, one row per PARENT, leaves the kernel.
 //   EPI_LEVEL  one level: (i, o, u) pre-activations = P + U_iou h~ with h~ the child sums; the epilogue adds
-//              S_j = sum_k f_jk c_k and finishes c_j = i u + S_j, h_j = o tanh(c_j).
+//              S_j and finishes c_j = i u + S_j, h_j = o tanh(c_j), and files the bf16 copy of h_j at its slot.
 //
-// gather_kernel is the bandwidth part of a level: one warp per node reads the h, G and c rows of its children
-// with coalesced 16-byte loads and produces the bf16 operand h~ (fp32 adds, rounded once) and S_j.
+// childsum_kernel produces the operand h~ of EPI_LEVEL: one warp per node adds the node's (contiguous) child rows.
 // The level loop is host-driven here (three launches per level); forests whose levels are too small for that
 // run the cooperative single-launch kernel of forward_small.cu instead.
 #include <cuda.h>
@@ -41,7 +44,7 @@ constexpr int GEMM1_THREADS = 224;  // warp 0: TMA producer, warps 1 and 6: MMA 
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;
 constexpr int TMEM_COLS = 512;  // two accumulator buffers of up to 256 columns
 
-enum { EPI_XPROJ = 0, EPI_LEVEL = 1, EPI_G = 2 };
+enum { EPI_XPROJ = 0, EPI_LEVEL = 1, EPI_F = 2 };
 
 struct TcArgs {
     const int32_t* child_ptr;
@@ -49,22 +52,43 @@ struct TcArgs {
     const int32_t* level_ptr;
     const int32_t* perm;
     int32_t* meta;
-    int32_t n_nodes, H, Hp;
+    int32_t n_nodes, n_edges, n_int_bound, H, Hp;
     const float* bias4;   // [Hp][4]
     float* P;             // [n_internal][4][Hp]   row = perm position - n_leaves, planes i, o, u, f
-    float* S;             // [n_internal][Hp]      sum_k f_jk c_k, row = perm position - n_leaves
+    float* S;             // [n_internal][Hp]      sum_k f_jk c_k, row = perm position - n_leaves (zeroed per call)
     __nv_bfloat16* hs;    // [n_internal][Hp]      child sums, row = perm position - n_leaves
-    __nv_bfloat16* hb;    // [n_nodes][Hp]         bf16 copy of h, row = perm position
-    float* G;             // [n_nodes][Hp]         U_f h, row = node id (row = perm position when p_tma is set)
+    __nv_bfloat16* hb;    // [n_nodes][Hp]         bf16 copy of h: row = slot of the node as a child (child_order), or
+                          //                       row = perm position (cooperative loop)
     float* h;
     float* c;
     int64_t ldh;
     int32_t vec_ok;       // h/c rows allow 16-byte accesses
-    const int32_t* inv;   // position of every node in level order
-    int32_t p_tma;        // rows in level order (P, the bf16 copy of leaf rows, G) leave through TMA stores; G is then
-                          // kept by position, not by node id
+    int32_t* inv;         // position of every node in level order
+    int32_t p_tma;        // rows in level order (P; the bf16 copy of leaf rows when it is kept by position) leave
+                          // through TMA stores
     int32_t issuers;      // MMA issuer warps of the lone-CTA GEMM: 1 (whole tile width) or 2 (half each)
+    // the child-ordered layout of the per-level launches
+    int32_t child_order;
+    int32_t* eoff;        // [n_internal + 1]  first slot of every internal node's children, row = position - n_leaves
+    int32_t* slot_of_pos; // [n_nodes]         slot of the node at a position in level order (-1: a root)
+    int32_t* slot_par;    // [n_edges]         row (position - n_leaves) of the parent that owns the slot
+    int32_t* slot_child;  // [n_edges]         node id of the child at the slot
+    int32_t debug;        // check every index against its array before following it
 };
+
+// JDB_FLAG_DEBUG_CHECKS: true if 0 <= v < bound.  Otherwise the first offender of the call is recorded in meta
+// (what, value, bound, where) and the caller skips the access.
+enum { CHECK_PERM = 1, CHECK_CHILD = 2, CHECK_POSITION = 3, CHECK_SLOT = 4, CHECK_PARENT_ROW = 5, CHECK_LEVEL_PTR = 6,
+       CHECK_EDGE_PTR = 7 };
+__device__ __forceinline__ bool dbg_ok(int32_t* meta, int what, long long v, long long bound, int where) {
+    if (v >= 0 && v < bound) return true;
+    if (atomicCAS(&meta[META_CHECK], 0, what) == 0) {
+        meta[META_CHECK + 1] = (int32_t)(v < -2147483647LL ? -2147483647LL : (v > 2147483647LL ? 2147483647LL : v));
+        meta[META_CHECK + 2] = (int32_t)(bound > 2147483647LL ? 2147483647LL : bound);
+        meta[META_CHECK + 3] = where;
+    }
+    return false;
+}
 
 // Where a tile sits.  The input projection walks the rows in level order and never mixes
 // leaves and internal nodes in a tile: leaf tiles need only the i, o, u blocks (192 of the 256 columns of a
@@ -106,14 +130,25 @@ constexpr int LEVEL_BN = 192;
 constexpr int LEVEL_STAGES = 3;
 constexpr int LEVEL_STAGE_BYTES = A_BYTES + LEVEL_BN * BK * 2;
 constexpr int GEMM_SMEM_LEVEL = LEVEL_STAGES * LEVEL_STAGE_BYTES + EPI_SCRATCH_BYTES + 1024;
-constexpr int GEMM_SMEM_STORE = GEMM_SMEM + 4 * EPI_STEP_FLOATS * 4;   // input projection and U_f GEMMs: one step buffer per warp
+constexpr int GEMM_SMEM_STORE = GEMM_SMEM + 4 * EPI_STEP_FLOATS * 4;   // input projection: one step buffer per warp
+// forget-gate GEMM: three full-width stages and a ring of three step buffers per warp, each two [32 rows][16 floats]
+// arrays (the parent's forget pre-activation and the child's c)
+constexpr int F_STEP_FLOATS = 2 * 32 * 16;
+constexpr int F_STAGES = 3;
+constexpr int F_SCRATCH_BYTES = 4 * EPI_RING * F_STEP_FLOATS * 4;
+constexpr int GEMM_SMEM_F = F_STAGES * STAGE_BYTES + F_SCRATCH_BYTES + 1024;
 static_assert(GEMM_SMEM_STORE <= 227 * 1024 - 256, "GEMM shared memory");
+static_assert(GEMM_SMEM_F <= 227 * 1024 - 256, "forget GEMM shared memory");
 static_assert(GEMM_SMEM_LEVEL <= 227 * 1024 - 256, "level GEMM shared memory");
 
 __device__ __forceinline__ int sw_off(int row, int chunk) { return row * 16 + ((chunk ^ ((row >> 1) & 3)) << 2); }
 
 __device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// the same through L1 (rows that many lanes of the CTA ask for again and again: a parent's row, once per child)
+__device__ __forceinline__ void cp_async16_ca_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -144,9 +179,11 @@ __device__ __forceinline__ void level_fetch(const TcArgs& a, const Tile& ti, int
 // HB_TILE: the bf16 copy is not stored here but collected, across the four steps of a tile, as a [32 rows][64 columns]
 // tile in the second half of the step buffer (128-byte rows, 16-byte chunk c of row r at chunk c ^ (r & 7)), which the
 // caller sends off as one TMA store.
+// hbr: rows of the bf16 copy that receive tile rows (lane >> 1) and (lane >> 1) + 16 of this warp (-1: none), when
+// the copy is stored here.
 template <bool HB_TILE = false>
 __device__ __forceinline__ void store_hc_step(const TcArgs& a, const Tile& ti, int quarter, int lane, int q, const int (&vs)[4],
-                                              const float (&cv)[16], const float (&hv)[16], float* sc) {
+                                              const int (&hbr)[2], const float (&cv)[16], const float (&hv)[16], float* sc) {
     const int lr = lane >> 2, lc = lane & 3;
 #pragma unroll
     for (int c4 = 0; c4 < 4; ++c4) {
@@ -192,9 +229,9 @@ __device__ __forceinline__ void store_hc_step(const TcArgs& a, const Tile& ti, i
     if (!HB_TILE) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {  // bf16 copy of h: 32 bytes per row, two lanes per row
-            const int r = (lane >> 1) + 16 * i, p = ti.row0 + quarter * 32 + r;
-            if (p < ti.row_end)
-                *reinterpret_cast<uint4*>(a.hb + (size_t)p * a.Hp + ti.n_tile * 64 + q * 16 + (lane & 1) * 8) =
+            const int r = (lane >> 1) + 16 * i;
+            if (hbr[i] >= 0)
+                *reinterpret_cast<uint4*>(a.hb + (size_t)hbr[i] * a.Hp + ti.n_tile * 64 + q * 16 + (lane & 1) * 8) =
                     *reinterpret_cast<const uint4*>(sc + 1024 + sw_off(r, lane & 1));
         }
     }
@@ -203,7 +240,7 @@ __device__ __forceinline__ void store_hc_step(const TcArgs& a, const Tile& ti, i
 
 // One 16-column step of a level tile for this warp's 32 rows: `sc` holds the step's P and S slices.
 __device__ __forceinline__ void level_step(const TcArgs& a, const Tile& ti, uint32_t taddr, int quarter, int lane, int q,
-                                           const int (&vs)[4], float* sc) {
+                                           const int (&vs)[4], const int (&hbr)[2], float* sc) {
     float gi[16], go[16], gu[16];
     tmem_ld16(taddr + q * 16, gi);
     tmem_ld16(taddr + 64 + q * 16, go);
@@ -225,13 +262,13 @@ __device__ __forceinline__ void level_step(const TcArgs& a, const Tile& ti, uint
         hv[4 * c4 + 3] = sigmoid_fast(go[4 * c4 + 3] + po.w) * tanh_fast(cv[4 * c4 + 3]);
     }
     __syncwarp();  // every lane has read its inputs: the arrays now carry the outputs
-    store_hc_step(a, ti, quarter, lane, q, vs, cv, hv, sc);
+    store_hc_step(a, ti, quarter, lane, q, vs, hbr, cv, hv, sc);
 }
 
 // x-projection step of a leaf tile: the cell finishes here (no children, so c = i u and h = o tanh(c)).
 template <bool HB_TILE>
 __device__ __forceinline__ void xproj_leaf_step(const TcArgs& a, const Tile& ti, uint32_t taddr, int quarter, int lane, int q,
-                                                const int (&vs)[4], float* sc) {
+                                                const int (&vs)[4], const int (&hbr)[2], float* sc) {
     const float4* bias4 = reinterpret_cast<const float4*>(a.bias4);
     float gi[16], go[16], gu[16];
     tmem_ld16(taddr + q * 16, gi);
@@ -247,7 +284,7 @@ __device__ __forceinline__ void xproj_leaf_step(const TcArgs& a, const Tile& ti,
         cv[i] = cc;
         hv[i] = sigmoid_fast(go[i] + b.y) * tanh_fast(cc);
     }
-    store_hc_step<HB_TILE>(a, ti, quarter, lane, q, vs, cv, hv, sc);
+    store_hc_step<HB_TILE>(a, ti, quarter, lane, q, vs, hbr, cv, hv, sc);
 }
 
 // x-projection step of a tile of internal nodes: the four biased pre-activations go to the planes of P.
@@ -329,57 +366,90 @@ __device__ __forceinline__ void xproj_internal_tile_tma(const TcArgs& a, const T
     __syncwarp();
 }
 
-// 64 columns of G = U_f h for this warp's 32 rows: 256 contiguous bytes per row, sixteen lanes per row.
-__device__ __forceinline__ void g_step(const TcArgs& a, const Tile& ti, uint32_t taddr, int lane, int qq, int vrow, float* sc) {
+// ---- epilogue of a forget-gate tile ---------------------------------------------------------------------------
+// Rows of the tile are edge slots, sorted by parent.  Per 16-column step a warp needs, for each of its 32 rows, the
+// parent's forget pre-activation P_f[parent] and the child's c_k: both arrive through the same kind of ring as the
+// level tile's P and S slices (four lanes per row, 16-byte asynchronous copies, two steps ahead).
+// pr, kd: parent row and child node id of tile rows (lane >> 2) + 8 i of this warp (-1: no such row).
+__device__ __forceinline__ void forget_fetch(const TcArgs& a, const Tile& ti, int lane, int q, const int (&pr)[4],
+                                             const int (&kd)[4], uint32_t buf, float* bufp) {
+    const int col = ti.n_tile * ti.bn + q * 16 + (lane & 3) * 4;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        float g[16];
-        tmem_ld16(taddr + qq * 64 + k * 16, g);
-        tmem_ld_wait();
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-            *reinterpret_cast<float4*>(sc + k * 512 + sw_off(lane, c4)) = make_float4(g[4 * c4], g[4 * c4 + 1], g[4 * c4 + 2], g[4 * c4 + 3]);
-    }
-    __syncwarp();
-    const int piece = lane & 15;
-#pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-        const int row = (lane >> 4) + 2 * i;
-        const int v = __shfl_sync(0xffffffffu, vrow, row);
-        if (v >= 0)
-            *reinterpret_cast<float4*>(a.G + (size_t)v * a.Hp + ti.n_tile * ti.bn + qq * 64 + piece * 4) =
-                *reinterpret_cast<const float4*>(sc + (piece >> 2) * 512 + sw_off(row, piece & 3));
-    }
-    __syncwarp();
-}
-
-// The same through the copy engine, with G kept by position: a warp's 32 rows x 64 columns are a plain box, staged as
-// two [32 rows][32 floats] halves in the tensor map's 128-byte swizzle and sent off by lane 0.  Rows past the level's
-// end belong to the next level, whose own launch writes them again before anything reads them.
-__device__ __forceinline__ void g_step_tma(const Tile& ti, const CUtensorMap* tmG, uint32_t taddr, int quarter, int lane, int qq,
-                                           float* sc) {
-    if (lane == 0) bulk_wait_read();  // the stores of the step before have read the buffer
-    __syncwarp();
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float g0[16], g1[16];
-        tmem_ld16(taddr + qq * 64 + half * 32, g0);
-        tmem_ld16(taddr + qq * 64 + half * 32 + 16, g1);
-        tmem_ld_wait();
-        uint8_t* row = reinterpret_cast<uint8_t*>(sc) + half * 4096 + lane * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const float* g = c < 4 ? &g0[4 * c] : &g1[4 * (c - 4)];
-            *reinterpret_cast<float4*>(row + ((c ^ (lane & 7)) << 4)) = make_float4(g[0], g[1], g[2], g[3]);
+    for (int i = 0; i < 4; ++i) {
+        const int row = (lane >> 2) + 8 * i;
+        const int o = sw_off(row, lane & 3);
+        const uint32_t d = buf + (uint32_t)o * 4;
+        const bool have = pr[i] >= 0;
+        cp_async16_ca_zfill(d, have ? a.P + ((size_t)pr[i] * 4 + 3) * a.Hp + col : a.P, have ? 16u : 0u);
+        const int left = have ? a.H - col : 0;   // columns of the child's c row from `col` on
+        if (left >= 4 && a.vec_ok) {
+            cp_async16_zfill(d + 2048, a.c + (int64_t)kd[i] * a.ldh + col, 16u);
+        } else if (left <= 0) {
+            cp_async16_zfill(d + 2048, a.P, 0u);
+        } else {  // ragged end of the row, or rows that are not 16-byte aligned
+            const float* src = a.c + (int64_t)kd[i] * a.ldh + col;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            v.x = __ldcg(src);
+            if (left > 1) v.y = __ldcg(src + 1);
+            if (left > 2) v.z = __ldcg(src + 2);
+            if (left > 3) v.w = __ldcg(src + 3);
+            *reinterpret_cast<float4*>(bufp + 512 + o) = v;
         }
     }
-    fence_proxy_async();
-    __syncwarp();
-    if (lane == 0) {
-        const int x = ti.n_tile * ti.bn + qq * 64, y = ti.row0 + quarter * 32;
-        tma_store_2d(tmG, smem_u32(sc), x, y);
-        tma_store_2d(tmG, smem_u32(sc) + 4096, x + 32, y);
-        bulk_commit();
+}
+
+// How this warp's 32 rows fall into runs of equal parent: distance of a lane from the first lane of its run, whether it
+// is the last lane of its run, and how many doubling steps the longest run needs.
+struct Runs {
+    int dist, steps;
+    bool last;
+};
+__device__ __forceinline__ Runs runs_of(int par, int lane) {
+    const int prev = __shfl_up_sync(0xffffffffu, par, 1), next = __shfl_down_sync(0xffffffffu, par, 1);
+    const unsigned heads = __ballot_sync(0xffffffffu, lane == 0 || prev != par);
+    Runs r;
+    r.dist = lane - (31 - __clz(heads & (0xffffffffu >> (31 - lane))));
+    r.last = lane == 31 || next != par;
+    const int longest = __reduce_max_sync(0xffffffffu, r.dist);
+    r.steps = longest == 0 ? 0 : 32 - __clz(longest);
+    return r;
+}
+
+// One 16-column step: f c_k for this lane's row, added up over the lanes of the same parent (an inclusive scan in
+// doubling steps that never crosses a run boundary), and the run totals added into S.  A parent whose children
+// straddle warps or tiles receives one contribution from each: S starts at zero and takes them by atomic adds.
+__device__ __forceinline__ void forget_step(const TcArgs& a, const Tile& ti, uint32_t taddr, int lane, int q, int par,
+                                            const Runs& runs, const float* sc) {
+    float g[16];
+    tmem_ld16(taddr + q * 16, g);
+    tmem_ld_wait();
+    float fc[16];
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+        const int o = sw_off(lane, c4);
+        const float4 pf = *reinterpret_cast<const float4*>(sc + o), ck = *reinterpret_cast<const float4*>(sc + 512 + o);
+        fc[4 * c4 + 0] = sigmoid_fast(pf.x + g[4 * c4 + 0]) * ck.x;
+        fc[4 * c4 + 1] = sigmoid_fast(pf.y + g[4 * c4 + 1]) * ck.y;
+        fc[4 * c4 + 2] = sigmoid_fast(pf.z + g[4 * c4 + 2]) * ck.z;
+        fc[4 * c4 + 3] = sigmoid_fast(pf.w + g[4 * c4 + 3]) * ck.w;
+    }
+    __syncwarp();  // every lane has read its inputs: the buffer may be refilled
+#pragma unroll 1
+    for (int k = 0; k < runs.steps; ++k) {
+        const int off = 1 << k;
+        const bool take = runs.dist >= off;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float up = __shfl_up_sync(0xffffffffu, fc[i], off);
+            if (take) fc[i] += up;
+        }
+    }
+    if (runs.last && par >= 0) {
+        float* dst = a.S + (size_t)par * a.Hp + ti.n_tile * ti.bn + q * 16;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * c4), "f"(fc[4 * c4]), "f"(fc[4 * c4 + 1]),
+                         "f"(fc[4 * c4 + 2]), "f"(fc[4 * c4 + 3]) : "memory");
     }
 }
 
@@ -389,7 +459,7 @@ __device__ __forceinline__ void g_step_tma(const Tile& ti, const CUtensorMap* tm
 // waits on its own copy of the accumulator barrier and releases the accumulator at the pair leader.
 // `scratch` is this CTA's epilogue shared memory (ring or step buffers of the four warps).
 template <int EPI, bool PAIR>
-__device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMap* tmP, const CUtensorMap* tmHB, const CUtensorMap* tmG,
+__device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMap* tmP, const CUtensorMap* tmHB,
                                                float* scratch, uint32_t tmem_base, uint64_t* bar_tfull,
                                                uint64_t* bar_tempty, volatile int* abort, int warp, int lane, int t0, int t_step,
                                                int total_tiles, int n_tiles, int lo, int hi, int bn, int n_leaves, int mt_leaf,
@@ -400,8 +470,10 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         if (PAIR) ti.row0 += rank * BM;
         return ti;
     };
+    // the verdict is taken over the whole warp: the accumulator loads that follow are warp-wide instructions
     auto wait_acc = [&](int acc, uint32_t phase) {
-        return PAIR ? mbar_wait_cluster(smem_u32(&bar_tfull[acc]), phase, abort) : mbar_wait(smem_u32(&bar_tfull[acc]), phase, abort);
+        const bool mine = PAIR ? mbar_wait_cluster(smem_u32(&bar_tfull[acc]), phase, abort) : mbar_wait(smem_u32(&bar_tfull[acc]), phase, abort);
+        return __all_sync(0xffffffffu, mine) != 0;
     };
     auto release_acc = [&](int acc) {
         tc_fence_before();
@@ -409,7 +481,20 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         else mbar_arrive(smem_u32(&bar_tempty[acc]));
     };
     const int quarter = warp & 3;           // TMEM lane quarter this warp may read
-    const int row = quarter * 32 + lane;    // accumulator row = TMEM lane
+    // node id of the row at position p (rows this lane stores), and the row of the bf16 copy that receives it
+    auto node_at = [&](int p, int row_end) {
+        if (p >= row_end) return -1;
+        const int v = a.perm[p];
+        if (a.debug && !dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, p)) return -1;
+        return v;
+    };
+    auto copy_row_at = [&](int p, int row_end) {
+        if (p >= row_end) return -1;
+        if (!a.child_order) return p;
+        const int sl = a.slot_of_pos[p];
+        if (a.debug && sl >= 0 && !dbg_ok(a.meta, CHECK_SLOT, sl, a.n_edges, p)) return -1;
+        return sl;
+    };
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -436,12 +521,11 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         int cur = 0;
         for (int t = t0; t < total_tiles && ok; t += t_step) {
             const Tile ti = tile_at(t);
-            int vs[4];  // node ids of the rows this lane stores
+            int vs[4], hbr[2];  // node ids of the rows this lane stores; rows of the bf16 copy
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int p = ti.row0 + quarter * 32 + (lane >> 2) + 8 * i;
-                vs[i] = p < ti.row_end ? a.perm[p] : -1;
-            }
+            for (int i = 0; i < 4; ++i) vs[i] = node_at(ti.row0 + quarter * 32 + (lane >> 2) + 8 * i, ti.row_end);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) hbr[i] = copy_row_at(ti.row0 + quarter * 32 + (lane >> 1) + 16 * i, ti.row_end);
             if (!wait_acc(acc, acc_phase)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
@@ -450,7 +534,68 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
                 fetch_next();                // into the buffer the previous step has just released
                 cp_async_wait<2>();          // this step's own copies have landed
                 __syncwarp();                // ... and so have the other lanes'
-                level_step(a, ti, taddr, quarter, lane, q, vs, ring + cur * EPI_STEP_FLOATS);
+                level_step(a, ti, taddr, quarter, lane, q, vs, hbr, ring + cur * EPI_STEP_FLOATS);
+                if (++cur == EPI_RING) cur = 0;
+            }
+            release_acc(acc);
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1u;
+        }
+        cp_async_wait<0>();
+    } else if (EPI == EPI_F) {
+        // rows are edge slots; the parent's forget pre-activation and the child's c arrive two steps ahead
+        float* ring = scratch + quarter * (EPI_RING * F_STEP_FLOATS);
+        const uint32_t ring_addr = smem_u32(ring);
+        const int steps = bn >> 4;
+        auto slot_rows = [&](const Tile& ti, int (&pr)[4], int (&kd)[4]) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int sl = ti.row0 + quarter * 32 + (lane >> 2) + 8 * i;
+                pr[i] = kd[i] = -1;
+                if (sl < ti.row_end) {
+                    pr[i] = a.slot_par[sl];
+                    kd[i] = a.slot_child[sl];
+                    if (a.debug && (!dbg_ok(a.meta, CHECK_PARENT_ROW, pr[i], a.n_int_bound, sl) ||
+                                    !dbg_ok(a.meta, CHECK_CHILD, kd[i], a.n_nodes, sl)))
+                        pr[i] = kd[i] = -1;
+                }
+            }
+        };
+        int f_t = t0, f_q = 0, f_buf = 0;
+        Tile f_ti = tile_at(f_t);
+        int f_pr[4], f_kd[4];
+        if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
+        auto fetch_next = [&]() {
+            if (f_t < total_tiles) {
+                forget_fetch(a, f_ti, lane, f_q, f_pr, f_kd, ring_addr + (uint32_t)f_buf * (F_STEP_FLOATS * 4), ring + f_buf * F_STEP_FLOATS);
+                if (++f_q == steps) {
+                    f_q = 0;
+                    f_t += t_step;
+                    f_ti = tile_at(f_t);
+                    if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
+                }
+            }
+            cp_async_commit();
+            if (++f_buf == EPI_RING) f_buf = 0;
+        };
+        fetch_next();
+        fetch_next();
+        int cur = 0;
+        for (int t = t0; t < total_tiles && ok; t += t_step) {
+            const Tile ti = tile_at(t);
+            const int sl = ti.row0 + quarter * 32 + lane;   // this lane's accumulator row
+            int par = sl < ti.row_end ? a.slot_par[sl] : -1;
+            if (a.debug && par >= 0 && !dbg_ok(a.meta, CHECK_PARENT_ROW, par, a.n_int_bound, sl)) par = -1;
+            const Runs runs = runs_of(par, lane);
+            if (!wait_acc(acc, acc_phase)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+            for (int q = 0; q < steps; ++q) {
+                fetch_next();
+                cp_async_wait<2>();
+                __syncwarp();
+                forget_step(a, ti, taddr, lane, q, par, runs, ring + cur * F_STEP_FLOATS);
                 if (++cur == EPI_RING) cur = 0;
             }
             release_acc(acc);
@@ -459,54 +604,45 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         }
         cp_async_wait<0>();
     } else {
-        // stores only: every step goes through one step buffer per warp to leave in coalesced pieces
+        // input projection: stores only; every step goes through one step buffer per warp to leave in coalesced pieces
         float* sc = scratch + quarter * EPI_STEP_FLOATS;
         for (int t = t0; t < total_tiles && ok; t += t_step) {
             const Tile ti = tile_at(t);
+            const bool leaf = ti.bn == 192;
             // node ids, fetched while the main loop of this tile is still running
-            int vs[4];
+            int vs[4], hbr[2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int p = ti.row0 + quarter * 32 + (lane >> 2) + 8 * i;
-                vs[i] = (EPI == EPI_XPROJ && ti.bn == 192 && p < ti.row_end) ? a.perm[p] : -1;
-            }
-            const int vrow = (EPI == EPI_G && ti.row0 + row < ti.row_end) ? a.perm[ti.row0 + row] : -1;
+            for (int i = 0; i < 4; ++i) vs[i] = leaf ? node_at(ti.row0 + quarter * 32 + (lane >> 2) + 8 * i, ti.row_end) : -1;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) hbr[i] = leaf ? copy_row_at(ti.row0 + quarter * 32 + (lane >> 1) + 16 * i, ti.row_end) : -1;
             if (!wait_acc(acc, acc_phase)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
-            if (EPI == EPI_XPROJ) {
-                if (ti.bn == 192) {
-                    if (a.p_tma) {
-                        // the bf16 copy of the tile's rows leaves as one TMA store (rows in level order: a plain box).
-                        // Rows of a partly filled last leaf tile belong to internal nodes, whose rows are written
-                        // again, with their values, by the level that evaluates them.
-                        if (lane == 0) bulk_wait_read();  // the store of the tile before has read the tile buffer
-                        __syncwarp();
+            if (leaf) {
+                if (a.p_tma && !a.child_order) {
+                    // the bf16 copy is kept by position: the tile's rows leave as one TMA store (a plain box).
+                    // Rows of a partly filled last leaf tile belong to internal nodes, whose rows are written
+                    // again, with their values, by the level that evaluates them.
+                    if (lane == 0) bulk_wait_read();  // the store of the tile before has read the tile buffer
+                    __syncwarp();
 #pragma unroll 1
-                        for (int q = 0; q < 4; ++q) xproj_leaf_step<true>(a, ti, taddr, quarter, lane, q, vs, sc);
-                        fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(tmHB, smem_u32(sc) + 4096, ti.n_tile * 64, ti.row0 + quarter * 32);
-                            bulk_commit();
-                        }
-                    } else {
-#pragma unroll 1
-                        for (int q = 0; q < 4; ++q) xproj_leaf_step<false>(a, ti, taddr, quarter, lane, q, vs, sc);
+                    for (int q = 0; q < 4; ++q) xproj_leaf_step<true>(a, ti, taddr, quarter, lane, q, vs, hbr, sc);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(tmHB, smem_u32(sc) + 4096, ti.n_tile * 64, ti.row0 + quarter * 32);
+                        bulk_commit();
                     }
                 } else {
-                    if (a.p_tma) {
-                        xproj_internal_tile_tma(a, ti, tmP, taddr, quarter, lane, n_leaves, sc);
-                    } else {
 #pragma unroll 1
-                        for (int q = 0; q < 4; ++q) xproj_internal_step(a, ti, taddr, quarter, lane, q, n_leaves, sc);
-                    }
+                    for (int q = 0; q < 4; ++q) xproj_leaf_step<false>(a, ti, taddr, quarter, lane, q, vs, hbr, sc);
                 }
             } else {
+                if (a.p_tma) {
+                    xproj_internal_tile_tma(a, ti, tmP, taddr, quarter, lane, n_leaves, sc);
+                } else {
 #pragma unroll 1
-                for (int qq = 0; qq < (ti.bn >> 6); ++qq) {
-                    if (a.p_tma) g_step_tma(ti, tmG, taddr, quarter, lane, qq, sc);
-                    else g_step(a, ti, taddr, lane, qq, vrow, sc);
+                    for (int q = 0; q < 4; ++q) xproj_internal_step(a, ti, taddr, quarter, lane, q, n_leaves, sc);
                 }
             }
             release_acc(acc);
@@ -518,13 +654,34 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
     if (!ok) *abort = 1;
 }
 
+// Row range of one level's launch: positions of the level's nodes (gate GEMM), or the slots of their children
+// (forget-gate GEMM).  An inconsistent range is recorded (debug checks) and made empty.
+template <int EPI>
+__device__ __forceinline__ void level_range(const TcArgs& a, int level, int n_leaves, int& lo, int& hi) {
+    lo = a.level_ptr[level];
+    hi = a.level_ptr[level + 1];
+    bool good = !a.debug || (dbg_ok(a.meta, CHECK_LEVEL_PTR, lo, (long long)a.n_nodes + 1, level) &&
+                             dbg_ok(a.meta, CHECK_LEVEL_PTR, hi, (long long)a.n_nodes + 1, level) &&
+                             dbg_ok(a.meta, CHECK_LEVEL_PTR, hi - lo, (long long)a.n_nodes + 1, level) &&
+                             dbg_ok(a.meta, CHECK_LEVEL_PTR, lo - n_leaves, (long long)a.n_int_bound + 1, level) &&
+                             dbg_ok(a.meta, CHECK_LEVEL_PTR, hi - n_leaves, (long long)a.n_int_bound + 1, level));
+    if (good && EPI == EPI_F) {
+        lo = a.eoff[lo - n_leaves];
+        hi = a.eoff[hi - n_leaves];
+        good = !a.debug || (dbg_ok(a.meta, CHECK_EDGE_PTR, lo, (long long)a.n_edges + 1, level) &&
+                            dbg_ok(a.meta, CHECK_EDGE_PTR, hi, (long long)a.n_edges + 1, level) &&
+                            dbg_ok(a.meta, CHECK_EDGE_PTR, hi - lo, (long long)a.n_edges + 1, level));
+    }
+    if (!good) lo = hi = 0;
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(GEMM1_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
-               const __grid_constant__ CUtensorMap tmHBs, const __grid_constant__ CUtensorMap tmG, TcArgs a, int level, int bn, int n_total, int kblocks) {
-    // the level GEMM trades one pipeline stage (its K is the hidden size: few blocks) for the epilogue's ring
-    constexpr int NST = EPI == EPI_LEVEL ? LEVEL_STAGES : STAGES;
+               const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
+    // the per-level GEMMs trade one pipeline stage (their K is the hidden size: few blocks) for the epilogue's ring
+    constexpr int NST = EPI == EPI_LEVEL ? LEVEL_STAGES : EPI == EPI_F ? F_STAGES : STAGES;
     constexpr int SB = EPI == EPI_LEVEL ? LEVEL_STAGE_BYTES : STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[NST], bar_empty[NST], bar_tfull[2], bar_tempty[2];
@@ -566,7 +723,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (EPI == EPI_XPROJ) {
         hi = a.n_nodes;
     } else if (level < n_levels) {
-        lo = a.level_ptr[level]; hi = a.level_ptr[level + 1];
+        level_range<EPI>(a, level, n_leaves, lo, hi);
         a_row_off = (EPI == EPI_LEVEL) ? -n_leaves : 0;
     }
     const int mt_leaf = EPI == EPI_XPROJ ? (n_leaves + BM - 1) / BM : 0;
@@ -640,7 +797,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!ok && lane == 0) *abort = 1;
         }
     } else if (warp >= 2 && warp <= 5) {
-        epilogue_warps<EPI, false>(a, &tmP, &tmHBs, &tmG, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST * SB), tmem_base,
+        epilogue_warps<EPI, false>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST * SB), tmem_base,
                                    bar_tfull, bar_tempty, abort, warp, lane, blockIdx.x, gridDim.x, total_tiles, n_tiles, lo, hi,
                                    bn, n_leaves, mt_leaf, 0);
     }
@@ -666,14 +823,15 @@ constexpr int STAGES2 = 6, STAGES2_LEVEL = 4;
 constexpr int STAGE2_BYTES = A_BYTES + B_BYTES_MAX / 2;
 constexpr int GEMM2_SMEM = STAGES2 * STAGE2_BYTES + 4 * EPI_STEP_FLOATS * 4 + 1024;
 constexpr int GEMM2_SMEM_LEVEL = STAGES2_LEVEL * STAGE2_BYTES + EPI_SCRATCH_BYTES + 1024;
+constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH_BYTES + 1024;
 static_assert(GEMM2_SMEM_LEVEL <= 227 * 1024 - 256, "pair level GEMM shared memory");
 
 template <int EPI>
 __global__ void __launch_bounds__(GEMM1_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
-               const __grid_constant__ CUtensorMap tmHBs, const __grid_constant__ CUtensorMap tmG, TcArgs a, int level, int bn, int n_total, int kblocks) {
-    constexpr int NST2 = EPI == EPI_LEVEL ? STAGES2_LEVEL : STAGES2;
+               const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
+    constexpr int NST2 = EPI == EPI_XPROJ ? STAGES2 : STAGES2_LEVEL;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[NST2], bar_empty[NST2], bar_tfull[2], bar_tempty[2];
     __shared__ uint32_t s_tmem_base;
@@ -693,7 +851,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         lo = 0; hi = a.n_nodes; a_row_off = 0;
     } else {
         if (level >= n_levels) return;  // uniform over the whole grid; nothing allocated, no cluster barrier yet
-        lo = a.level_ptr[level]; hi = a.level_ptr[level + 1];
+        level_range<EPI>(a, level, n_leaves, lo, hi);
         a_row_off = (EPI == EPI_LEVEL) ? -n_leaves : 0;
     }
     constexpr int TM2 = 2 * BM;
@@ -716,7 +874,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
     }
-    if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), TMEM_COLS);
+    if (warp == 1) tmem_alloc<2>(smem_u32(&s_tmem_base), TMEM_COLS);  // one warp of each CTA of the pair, together
     tc_fence_before();
     __syncthreads();
     cluster_sync();  // the peer's barriers exist before anything is sent to them
@@ -792,7 +950,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (!ok && lane == 0) *abort = 1;
         }
     } else if (warp >= 2 && warp <= 5) {
-        epilogue_warps<EPI, true>(a, &tmP, &tmHBs, &tmG, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST2 * STAGE2_BYTES),
+        epilogue_warps<EPI, true>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST2 * STAGE2_BYTES),
                                   tmem_base, bar_tfull, bar_tempty, abort, warp, lane, pair, n_pairs, total_tiles, n_tiles, lo, hi,
                                   bn, n_leaves, mt_leaf, (int)rank);
     }
@@ -805,81 +963,180 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     cluster_sync();  // nothing of the peer (commits, arrivals) is still on its way to this CTA's memory
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (warp == 1) tmem_dealloc<2>(tmem_base, TMEM_COLS);
 }
 
-// The bandwidth part of one level, one warp per node: h~_j = sum_k h_k (fp32 adds in CSR order, rounded to
-// bf16 once) and S_j = sum_k sig(P_f[j] + G_k) * c_k.  Lanes run along the hidden dimension, so every child row
-// is read with coalesced 16-byte loads; two children are in flight per lane.
-__device__ __forceinline__ float4 ld4_guard(const float* row, int j, int H, int vec_ok) {
-    if (vec_ok && j + 4 <= H) return __ldcg(reinterpret_cast<const float4*>(row + j));
-    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (j < H) r.x = __ldcg(row + j);
-    if (j + 1 < H) r.y = __ldcg(row + j + 1);
-    if (j + 2 < H) r.z = __ldcg(row + j + 2);
-    if (j + 3 < H) r.w = __ldcg(row + j + 3);
-    return r;
-}
-
-__global__ void __launch_bounds__(256, 2) gather_kernel(TcArgs a, int level) {
+// The operand of a level's gate GEMM, one warp per node: h~_j = sum_k bf16(h_k), fp32 adds in child-list order,
+// rounded to bf16 once.  The child rows of a node are consecutive rows of the child-ordered copy, and the nodes of a
+// level own consecutive runs of them, so the kernel streams one contiguous range with 16-byte loads.
+__global__ void __launch_bounds__(256, 4) childsum_kernel(TcArgs a, int level) {
     griddep_wait();
     griddep_launch();
     const int n_levels = a.meta[META_N_LEVELS];
     if (level >= n_levels) return;
-    const int lo = a.level_ptr[level], hi = a.level_ptr[level + 1], n_leaves = a.level_ptr[1];
+    const int n_leaves = a.level_ptr[1];
+    int lo, hi;
+    level_range<EPI_LEVEL>(a, level, n_leaves, lo, hi);
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int pieces = a.Hp >> 3;  // 16-byte pieces of a row
     for (int pos = lo + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); pos < hi; pos += warps) {
-        const int v = a.perm[pos];
-        const int e0 = a.child_ptr[v], e1 = a.child_ptr[v + 1];
         const size_t r = (size_t)(pos - n_leaves);
-        const float* pf = a.P + r * 4 * a.Hp + 3 * a.Hp;
-        // 512 columns per pass: a lane holds four 16-byte pieces 128 columns apart, so the twelve loads of a
-        // child (h, c, G pieces) are all in flight together
-        for (int jb = 0; jb < a.Hp; jb += 512) {
-            float4 p[4], hs[4], sv[4];
+        int e0 = a.eoff[r], e1 = a.eoff[r + 1];
+        if (a.debug && (!dbg_ok(a.meta, CHECK_EDGE_PTR, e0, (long long)a.n_edges + 1, pos) ||
+                        !dbg_ok(a.meta, CHECK_EDGE_PTR, e1, (long long)a.n_edges + 1, pos) ||
+                        !dbg_ok(a.meta, CHECK_EDGE_PTR, e1 - e0, (long long)a.n_edges + 1, pos)))
+            e0 = e1 = 0;
+        // 1024 columns per pass: a lane holds four 16-byte pieces 256 columns apart
+        for (int pb = 0; pb < pieces; pb += 128) {
+            float acc[4][8];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                const int j = jb + m * 128 + lane * 4;
-                hs[m] = sv[m] = p[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (j < a.H) p[m] = __ldcg(reinterpret_cast<const float4*>(pf + j));
-            }
-            for (int e = e0; e < e1; ++e) {
-                const int k = a.child_idx[e];
-                const float* hk = a.h + (int64_t)k * a.ldh;
-                const float* ck = a.c + (int64_t)k * a.ldh;
-                const float* gk = a.G + (size_t)(a.p_tma ? a.inv[k] : k) * a.Hp;
-                float4 hh[4], cc[4], gg[4];
+            for (int m = 0; m < 4; ++m)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[m][i] = 0.f;
+            const uint4* src = reinterpret_cast<const uint4*>(a.hb + (size_t)e0 * a.Hp) + pb + lane;
+            for (int e = e0; e < e1; ++e, src += pieces) {
+                uint4 w[4];
+#pragma unroll
+                for (int m = 0; m < 4; ++m) w[m] = (pb + m * 32 + lane < pieces) ? __ldcg(src + m * 32) : make_uint4(0, 0, 0, 0);
 #pragma unroll
                 for (int m = 0; m < 4; ++m) {
-                    const int j = jb + m * 128 + lane * 4;
-                    hh[m] = cc[m] = gg[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (j < a.H) {
-                        hh[m] = ld4_guard(hk, j, a.H, a.vec_ok);
-                        cc[m] = ld4_guard(ck, j, a.H, a.vec_ok);
-                        gg[m] = __ldcg(reinterpret_cast<const float4*>(gk + j));
+                    const uint32_t u[4] = {w[m].x, w[m].y, w[m].z, w[m].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        acc[m][2 * i] += __uint_as_float(u[i] << 16);
+                        acc[m][2 * i + 1] += __uint_as_float(u[i] & 0xffff0000u);
                     }
                 }
-#pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    hs[m].x += hh[m].x; hs[m].y += hh[m].y; hs[m].z += hh[m].z; hs[m].w += hh[m].w;
-                    sv[m].x = fmaf(sigmoid_fast(p[m].x + gg[m].x), cc[m].x, sv[m].x);
-                    sv[m].y = fmaf(sigmoid_fast(p[m].y + gg[m].y), cc[m].y, sv[m].y);
-                    sv[m].z = fmaf(sigmoid_fast(p[m].z + gg[m].z), cc[m].z, sv[m].z);
-                    sv[m].w = fmaf(sigmoid_fast(p[m].w + gg[m].w), cc[m].w, sv[m].w);
-                }
             }
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const int j = jb + m * 128 + lane * 4;
-                if (j >= a.Hp) continue;
-                __nv_bfloat162 p0 = __floats2bfloat162_rn(hs[m].x, hs[m].y), p1 = __floats2bfloat162_rn(hs[m].z, hs[m].w);
-                uint2 w;
-                w.x = *reinterpret_cast<uint32_t*>(&p0);
-                w.y = *reinterpret_cast<uint32_t*>(&p1);
-                *reinterpret_cast<uint2*>(a.hs + r * a.Hp + j) = w;
-                *reinterpret_cast<float4*>(a.S + r * a.Hp + j) = sv[m];
+                if (pb + m * 32 + lane >= pieces) continue;
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    __nv_bfloat162 p2 = __floats2bfloat162_rn(acc[m][2 * i], acc[m][2 * i + 1]);
+                    o[i] = *reinterpret_cast<uint32_t*>(&p2);
+                }
+                reinterpret_cast<uint4*>(a.hs + r * a.Hp)[pb + m * 32 + lane] = make_uint4(o[0], o[1], o[2], o[3]);
             }
+        }
+    }
+}
+
+// ---- the child-ordered layout ----------------------------------------------------------------------------------
+// Edge slots: the children of the internal node at position p (row r = p - n_leaves) own slots eoff[r] .. eoff[r+1]-1 in
+// child-list order, eoff being the running sum of the child counts over the rows.  Three small kernels: counts and a
+// scan inside blocks of 1024 rows, a scan of the block totals, and the fill of the per-slot tables.
+constexpr int SCAN_TB = 1024;
+
+__global__ void __launch_bounds__(SCAN_TB) edge_count_kernel(TcArgs a, int32_t* block_sum) {
+    __shared__ int wsum[32];
+    griddep_wait();
+    griddep_launch();
+    const int n_levels = a.meta[META_N_LEVELS];
+    const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
+    const int n_int = a.n_nodes - n_leaves;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int r = blockIdx.x * SCAN_TB + threadIdx.x;
+    if (blockIdx.x * SCAN_TB > n_int) return;  // the block holds none of the rows 0 .. n_int
+    int cnt = 0;
+    if (r < n_int) {
+        const int v = a.perm[n_leaves + r];
+        if (!a.debug || dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, n_leaves + r)) cnt = a.child_ptr[v + 1] - a.child_ptr[v];
+        if (a.debug && !dbg_ok(a.meta, CHECK_EDGE_PTR, cnt, (long long)a.n_edges + 1, n_leaves + r)) cnt = 0;
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) wsum[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+        int t = wsum[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, t, o);
+            if (lane >= o) t += y;
+        }
+        wsum[lane] = t;
+    }
+    __syncthreads();
+    if (w > 0) incl += wsum[w - 1];
+    if (r <= n_int) a.eoff[r] = incl - cnt;  // exclusive, inside the block (row n_int: the block's running total so far)
+    if (threadIdx.x == SCAN_TB - 1) block_sum[blockIdx.x] = incl;
+}
+
+__global__ void __launch_bounds__(SCAN_TB) edge_scan_kernel(TcArgs a, int32_t* block_sum, int n_blocks_bound) {
+    __shared__ int wsum[32];
+    __shared__ int carry_s;
+    griddep_wait();
+    griddep_launch();
+    const int n_levels = a.meta[META_N_LEVELS];
+    const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
+    const int n_int = a.n_nodes - n_leaves;
+    int n_blocks = n_int / SCAN_TB + 1;  // blocks that hold a row 0 .. n_int
+    if (n_blocks > n_blocks_bound) n_blocks = n_blocks_bound;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    for (int base = 0; base < n_blocks; base += SCAN_TB) {
+        const int i = base + threadIdx.x;
+        const int x = i < n_blocks ? block_sum[i] : 0;
+        int incl = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        if (lane == 31) wsum[w] = incl;
+        __syncthreads();
+        if (w == 0) {
+            int t = wsum[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, t, o);
+                if (lane >= o) t += y;
+            }
+            wsum[lane] = t;
+        }
+        __syncthreads();
+        if (w > 0) incl += wsum[w - 1];
+        const int carry = carry_s;
+        if (i < n_blocks) block_sum[i] = incl - x + carry;  // exclusive over the blocks
+        __syncthreads();
+        if (threadIdx.x == SCAN_TB - 1) carry_s = carry + incl;
+        __syncthreads();
+    }
+}
+
+// One warp per internal node: finishes eoff and files every child under its slot.
+__global__ void __launch_bounds__(256) edge_fill_kernel(TcArgs a, const int32_t* block_sum) {
+    griddep_wait();
+    griddep_launch();
+    const int n_levels = a.meta[META_N_LEVELS];
+    const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
+    const int n_int = a.n_nodes - n_leaves;
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r <= n_int; r += warps) {
+        const int e0 = a.eoff[r] + block_sum[r / SCAN_TB];
+        __syncwarp();
+        if (lane == 0) a.eoff[r] = e0;
+        if (r == n_int) continue;
+        const int v = a.perm[n_leaves + r];
+        if (a.debug && !dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, n_leaves + r)) continue;
+        const int c0 = a.child_ptr[v], cnt = a.child_ptr[v + 1] - c0;
+        for (int i = lane; i < cnt; i += 32) {
+            const int k = a.child_idx[c0 + i], sl = e0 + i;
+            if (a.debug && (!dbg_ok(a.meta, CHECK_CHILD, k, a.n_nodes, v) || !dbg_ok(a.meta, CHECK_SLOT, sl, a.n_edges, v))) continue;
+            const int kp = a.inv[k];
+            if (a.debug && !dbg_ok(a.meta, CHECK_POSITION, kp, a.n_nodes, k)) continue;
+            a.slot_par[sl] = r;
+            a.slot_child[sl] = k;
+            a.slot_of_pos[kp] = sl;
         }
     }
 }
@@ -891,13 +1148,14 @@ __global__ void __launch_bounds__(256, 2) gather_kernel(TcArgs a, int level) {
 __global__ void __launch_bounds__(256) level_order_x_kernel(const void* __restrict__ x, int is_bf16, int64_t ldx,
                                                             const int32_t* __restrict__ perm, int N, int D, int Dp,
                                                             int vec_ok, __nv_bfloat16* __restrict__ out,
-                                                            int32_t* __restrict__ inv) {
+                                                            int32_t* __restrict__ inv, int32_t* meta, int debug) {
     griddep_wait();
     griddep_launch();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     for (int pos = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; pos < N; pos += warps) {
         const int64_t v = perm[pos];
+        if (debug && !dbg_ok(meta, CHECK_PERM, v, N, pos)) continue;
         if (inv && lane == 0) inv[v] = pos;  // where the node sits in level order
         __nv_bfloat16* dst = out + (size_t)pos * Dp;
         if (vec_ok) {  // bf16 source, 16-byte aligned rows
@@ -990,31 +1248,39 @@ bool make_tmap_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t col
     return r == CUDA_SUCCESS;
 }
 
-// Which GEMMs run as CTA pairs (cta_group::2) when they have enough 256-row tiles: a bit mask from JDB_GEMM_PAIR
-// (1 input projection, 2 level GEMM, 4 U_f GEMM).  Default 4: the U_f GEMM, whose epilogue only stores, gains from
-// the pair reading half of B per SM; the projection, with its heavier epilogue, does not.
-int pair_mask() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("JDB_GEMM_PAIR");
-        v = e ? (atoi(e) & 7) : 4;
+// The switches of one forward call (jdb_opts.tuning, or the defaults with the environment's overrides, read at every
+// call so that nothing depends on what an earlier call saw).
+//   pair_mask  which GEMMs run as CTA pairs (cta_group::2) when they have enough 256-row tiles: 1 input projection,
+//              2 level GEMM, 4 forget-gate GEMM.  Default 4: the forget-gate GEMM gains from the pair reading half of
+//              B per SM; the projection, with its heavier epilogue, does not.
+//   pdl        programmatic dependent launch of the forward kernels (each waits for its predecessor inside the
+//              kernel, after its own set-up)
+struct Tuning {
+    int pair_mask, issuers;
+    bool pdl, p_tma;
+};
+Tuning resolve_tuning(int32_t t) {
+    Tuning r;
+    if (t & JDB_TUNE_SET) {
+        r.pair_mask = ((t & JDB_TUNE_PAIR_XPROJ) ? 1 : 0) | ((t & JDB_TUNE_PAIR_LEVEL) ? 2 : 0) | ((t & JDB_TUNE_PAIR_FORGET) ? 4 : 0);
+        r.issuers = (t & JDB_TUNE_TWO_ISSUERS) ? 2 : 1;
+        r.pdl = !(t & JDB_TUNE_NO_PDL);
+        r.p_tma = !(t & JDB_TUNE_PLAIN_STORES);
+        return r;
     }
-    return v;
-}
-
-// Programmatic dependent launch of the forward kernels (each waits for its predecessor inside the kernel, after its
-// own set-up): on unless JDB_PDL=0 is set in the environment.
-bool pdl_mode() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("JDB_PDL");
-        v = (e && e[0] == '0') ? 0 : 1;
-    }
-    return v == 1;
+    const char* e = getenv("JDB_GEMM_PAIR");
+    r.pair_mask = e ? (atoi(e) & 7) : 4;
+    e = getenv("JDB_GEMM_ISSUERS");
+    r.issuers = (e && e[0] == '2') ? 2 : 1;
+    e = getenv("JDB_PDL");
+    r.pdl = !(e && e[0] == '0');
+    e = getenv("JDB_P_TMA");
+    r.p_tma = !(e && e[0] == '0');
+    return r;
 }
 
 template <class... KArgs, class... Args>
-cudaError_t launch_behind(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+cudaError_t launch_behind(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -1024,7 +1290,7 @@ cudaError_t launch_behind(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_mode() ? 1 : 0;
+    cfg.numAttrs = pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -1061,22 +1327,48 @@ jdb_status tc_pack_weights_enqueue(const float* W, const float* U, const float* 
     return JDB_OK;
 }
 
+namespace {
+// carving of the forward workspace (the same walk sizes it and hands out the pieces)
+struct TcWorkspace {
+    float* P;
+    __nv_bfloat16* hs;
+    float* S;
+    __nv_bfloat16* hb;
+    __nv_bfloat16* xb;
+    int32_t *inv, *eoff, *slot_of_pos, *slot_par, *slot_child, *block_sum;
+    size_t s_bytes, slot_of_pos_bytes, total;
+    int n_scan_blocks;
+};
+TcWorkspace carve_tc_ws(void* ws, int32_t n_nodes, int32_t n_internal_bound, int32_t D, int Hp) {
+    const size_t n = (size_t)(n_nodes > 0 ? n_nodes : 1), ni = (size_t)(n_internal_bound > 0 ? n_internal_bound : 1);
+    char* p = (char*)ws;
+    auto take = [&](size_t bytes) { char* q = p; p += align_up(bytes, 256); return q; };
+    TcWorkspace w{};
+    w.P = (float*)take(ni * Hp * 4 * sizeof(float));
+    w.hs = (__nv_bfloat16*)take(ni * Hp * 2);
+    w.s_bytes = ni * Hp * sizeof(float);
+    w.S = (float*)take(w.s_bytes);
+    w.hb = (__nv_bfloat16*)take(n * Hp * 2);
+    w.xb = (__nv_bfloat16*)take(n * (size_t)((D + 7) / 8 * 8) * 2);
+    w.inv = (int32_t*)take(n * sizeof(int32_t));
+    w.eoff = (int32_t*)take((ni + 1 + SCAN_TB) * sizeof(int32_t));
+    w.slot_of_pos_bytes = n * sizeof(int32_t);
+    w.slot_of_pos = (int32_t*)take(w.slot_of_pos_bytes);
+    w.slot_par = (int32_t*)take(n * sizeof(int32_t));
+    w.slot_child = (int32_t*)take(n * sizeof(int32_t));
+    w.n_scan_blocks = (int)(ni / SCAN_TB + 1);
+    w.block_sum = (int32_t*)take((size_t)w.n_scan_blocks * sizeof(int32_t));
+    w.total = (size_t)(p - (char*)ws);
+    return w;
+}
+}  // namespace
+
 size_t forward_tc_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D, int32_t H) {
-    TcPackLayout L = tc_pack_layout(D, H);
-    size_t n = (size_t)(n_nodes > 0 ? n_nodes : 1), ni = (size_t)(n_internal_bound > 0 ? n_internal_bound : 1);
-    size_t bytes = 0;
-    bytes += align_up(ni * L.Hp * 4 * sizeof(float), 256);           // P
-    bytes += align_up(ni * L.Hp * 2, 256);                           // hs
-    bytes += align_up(ni * L.Hp * sizeof(float), 256);               // S
-    bytes += align_up(n * L.Hp * 2, 256);                            // hb
-    bytes += align_up(n * L.Hp * sizeof(float), 256);                // G
-    bytes += align_up(n * (size_t)((D + 7) / 8 * 8) * 2, 256);       // converted x (when needed)
-    bytes += align_up(n * sizeof(int32_t), 256);                     // position of every node in level order
-    return bytes;
+    return carve_tc_ws(nullptr, n_nodes, n_internal_bound, D, tc_pack_layout(D, H).Hp).total;
 }
 
 jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int n_levels, int n_internal_bound,
-                              void* ws, bool use_small, int n_wide, uint64_t timeout_ns, cudaStream_t st) {
+                              void* ws, bool use_small, uint64_t timeout_ns, cudaStream_t st) {
     const int N = fa.n_nodes, D = fa.D, H = fa.H;
     TcPackLayout L = tc_pack_layout(D, H);
     const int Hp = L.Hp;
@@ -1085,68 +1377,54 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     if (!di) return JDB_ERR_CUDA;
     const int n_sm = di->n_sm;
 
-    size_t n = (size_t)N, ni = (size_t)(n_internal_bound > 0 ? n_internal_bound : 1);
-    char* p = (char*)ws;
-    auto take = [&](size_t bytes) { char* q = p; p += align_up(bytes, 256); return q; };
-    float* P = (float*)take(ni * Hp * 4 * sizeof(float));
-    __nv_bfloat16* hs = (__nv_bfloat16*)take(ni * Hp * 2);
-    float* S = (float*)take(ni * Hp * sizeof(float));
-    __nv_bfloat16* hb = (__nv_bfloat16*)take(n * Hp * 2);
-    float* G = (float*)take(n * Hp * sizeof(float));
+    const size_t n = (size_t)N, ni = (size_t)(n_internal_bound > 0 ? n_internal_bound : 1);
+    const TcWorkspace w = carve_tc_ws(ws, N, n_internal_bound, D, Hp);
     const int Dp = (D + 7) / 8 * 8;
-    __nv_bfloat16* xb = (__nv_bfloat16*)take(n * (size_t)Dp * 2);
-    int32_t* inv = (int32_t*)take(n * sizeof(int32_t));
 
     const char* pk = (const char*)packed_tc;
     TcArgs a{};
     a.child_ptr = fa.child_ptr; a.child_idx = fa.child_idx; a.level_ptr = fa.level_ptr; a.perm = fa.perm;
-    a.meta = fa.meta; a.n_nodes = N; a.H = H; a.Hp = Hp;
+    a.meta = fa.meta; a.n_nodes = N; a.n_edges = fa.n_edges; a.n_int_bound = (int32_t)ni; a.H = H; a.Hp = Hp;
     a.bias4 = (const float*)(pk + L.off_bias);
-    a.P = P; a.S = S; a.hs = hs; a.hb = hb; a.G = G; a.inv = inv; a.h = fa.h; a.c = fa.c; a.ldh = fa.ldh;
+    a.P = w.P; a.S = w.S; a.hs = w.hs; a.hb = w.hb; a.inv = w.inv; a.h = fa.h; a.c = fa.c; a.ldh = fa.ldh;
     a.vec_ok = (fa.ldh % 4 == 0) && (((uintptr_t)fa.h & 15) == 0) && (((uintptr_t)fa.c & 15) == 0);
-    {
-        const char* e = getenv("JDB_GEMM_ISSUERS");
-        a.issuers = (e && e[0] == '2') ? 2 : 1;
-    }
+    a.child_order = use_small ? 0 : 1;
+    a.eoff = w.eoff; a.slot_of_pos = w.slot_of_pos; a.slot_par = w.slot_par; a.slot_child = w.slot_child;
+    a.debug = fa.debug;
+    const Tuning tune = resolve_tuning(fa.tuning);
+    a.issuers = tune.issuers;
+    a.p_tma = tune.p_tma ? 1 : 0;
 
     // x goes into level order (and bf16) once; the copy reads 16-byte pieces when x is bf16 with aligned rows
     const int x_vec = fa.x_is_bf16 && (fa.ldx % 8 == 0) && (((uintptr_t)fa.x & 15) == 0);
-    const void* xsrc = xb;
-    const uint64_t xld = (uint64_t)Dp;
     // CTA pairs pay off once there are enough 256-row tiles to keep every pair busy; below that the lone-CTA
     // kernel has the shorter tail.  In pair mode every CTA loads half of a B tile, so the B maps have half-height boxes.
     const bool big = !use_small && (long long)N >= 2LL * BM * n_sm;
-    const bool pair_x = big && (pair_mask() & 1), pair_l = big && (pair_mask() & 2), pair_g = big && (pair_mask() & 4);
-    // in pair mode each CTA loads half of the B tile's rows
+    const bool pair_x = big && (tune.pair_mask & 1), pair_l = big && (tune.pair_mask & 2), pair_f = big && (tune.pair_mask & 4);
     const uint32_t bdiv = pair_x ? 2 : 1, bdiv_l = pair_l ? 2 : 1;
-    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmUf, tmUfH, tmP, tmHBs, tmG;
-    const int bng = g_bn(Hp);
+    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmUf, tmUfH, tmP, tmHBs;
+    const int bnf = g_bn(Hp);
     // W is read through a full box and a leaf box (i, o, u blocks only)
-    bool ok = make_tmap(&tmX, xsrc, n, (uint64_t)D, xld, BM) &&
+    bool ok = make_tmap(&tmX, w.xb, n, (uint64_t)D, (uint64_t)Dp, BM) &&
               make_tmap(&tmW, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 256 / bdiv) &&
               make_tmap(&tmWl, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 192 / bdiv);
-    if (ok && (!use_small || n_wide > 0))   // the per-level launches read their operands through four more maps
-        ok = make_tmap(&tmHS, hs, ni, (uint64_t)Hp, (uint64_t)Hp, BM) &&
+    if (ok && !use_small)   // the per-level launches read their operands through five more maps
+        ok = make_tmap(&tmHS, w.hs, ni, (uint64_t)Hp, (uint64_t)Hp, BM) &&
              make_tmap(&tmUiou, pk + L.off_Uiou, (uint64_t)3 * Hp, (uint64_t)Hp, (uint64_t)Hp, 192 / bdiv_l) &&
-             make_tmap(&tmHB, hb, n, (uint64_t)Hp, (uint64_t)Hp, BM) &&
-             make_tmap(&tmUf, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bng) &&
-             make_tmap(&tmUfH, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bng / 2);
-    ok = ok && make_tmap_f32(&tmP, P, ni, (uint64_t)4 * Hp, (uint64_t)4 * Hp) &&
-         make_tmap(&tmHBs, hb, n, (uint64_t)Hp, (uint64_t)Hp, 32) &&  // store boxes: 64 columns x one warp's 32 rows
-         make_tmap_f32(&tmG, G, n, (uint64_t)Hp, (uint64_t)Hp);
+             make_tmap(&tmHB, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, BM) &&
+             make_tmap(&tmUf, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bnf) &&
+             make_tmap(&tmUfH, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bnf / 2);
+    ok = ok && make_tmap_f32(&tmP, w.P, ni, (uint64_t)4 * Hp, (uint64_t)4 * Hp) &&
+         make_tmap(&tmHBs, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, 32);  // store boxes: 64 columns x one warp's 32 rows
     if (!ok) return JDB_ERR_UNSUPPORTED;
-    {
-        const char* e = getenv("JDB_P_TMA");  // rows of P through TMA stores: on unless JDB_P_TMA=0
-        a.p_tma = (e && e[0] == '0') ? 0 : 1;
-    }
 
     if (!(di->attr_mask & ATTR_GEMM_TC)) {
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_XPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_STORE));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_LEVEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_LEVEL));
-        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_G>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_STORE));
+        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_F>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_F));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_XPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_LEVEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM_LEVEL));
-        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_G>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM));
+        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_F>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM_F));
         di->attr_mask |= ATTR_GEMM_TC;
     }
 
@@ -1160,24 +1438,22 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     auto launch = [&](int epi, const CUtensorMap& tA, const CUtensorMap& tB_full, const CUtensorMap& tBl, long long rows_bound,
                       int level, int bn, int n_total, int kblocks) -> jdb_status {
         const int n_tiles = n_total / bn;
-        // the U_f GEMM decides launch by launch: pairs pay off from about 32 tiles per pair on (measured: they gain
-        // on the 1.4 M leaf rows of the wide forest and lose on 70 k rows)
+        // the forget-gate GEMM decides launch by launch: pairs pay off from about 32 tiles per pair on
         const long long tiles2 = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles;
-        const bool pair = epi == EPI_XPROJ ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_g && tiles2 >= 32LL * (n_sm / 2));
-        const CUtensorMap& tB = (epi == EPI_G && pair) ? tmUfH : tB_full;
+        const bool pair = epi == EPI_XPROJ ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_f && tiles2 >= 32LL * (n_sm / 2));
+        const CUtensorMap& tB = (epi == EPI_F && pair) ? tmUfH : tB_full;
         if (!pair) {
             const int grid = gemm_grid(rows_bound, n_tiles);
-            if (epi == EPI_XPROJ) JDB_CUDA_TRY(launch_behind(gemm_tc_kernel<EPI_XPROJ>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
-            else if (epi == EPI_LEVEL) JDB_CUDA_TRY(launch_behind(gemm_tc_kernel<EPI_LEVEL>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_LEVEL, st, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
-            else JDB_CUDA_TRY(launch_behind(gemm_tc_kernel<EPI_G>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
+            if (epi == EPI_XPROJ) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+            else if (epi == EPI_LEVEL) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_LEVEL>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_LEVEL, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+            else JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_F>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_F, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
             return JDB_OK;
         }
-        long long tiles = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles;
-        int pairs = (int)(tiles < n_sm / 2 ? (tiles > 0 ? tiles : 1) : n_sm / 2);
+        int pairs = (int)(tiles2 < n_sm / 2 ? (tiles2 > 0 ? tiles2 : 1) : n_sm / 2);
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(2 * pairs);
         cfg.blockDim = dim3(GEMM1_THREADS);
-        cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : GEMM2_SMEM;
+        cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : epi == EPI_F ? GEMM2_SMEM_F : GEMM2_SMEM;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1187,10 +1463,10 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = pdl_mode() ? 2 : 1;
-        if (epi == EPI_XPROJ) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_XPROJ>, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
-        else if (epi == EPI_LEVEL) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_LEVEL>, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
-        else JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_G>, tA, tB, tBl, tmP, tmHBs, tmG, a, level, bn, n_total, kblocks));
+        cfg.numAttrs = tune.pdl ? 2 : 1;
+        if (epi == EPI_XPROJ) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_XPROJ>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+        else if (epi == EPI_LEVEL) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_LEVEL>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+        else JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_F>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
         return JDB_OK;
     };
 
@@ -1199,29 +1475,31 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     {
         const long long want = ((long long)N + 7) / 8;
         const int blocks = (int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16);
-        JDB_CUDA_TRY(launch_behind(level_order_x_kernel, dim3(blocks), dim3(256), 0, st, fa.x, (int)fa.x_is_bf16, fa.ldx, fa.perm, N, D, Dp,
-                                   (int)x_vec, xb, inv));
+        JDB_CUDA_TRY(launch_behind(tune.pdl, level_order_x_kernel, dim3(blocks), dim3(256), 0, st, fa.x, (int)fa.x_is_bf16, fa.ldx, fa.perm, N, D, Dp,
+                                   (int)x_vec, w.xb, w.inv, fa.meta, (int)fa.debug));
+    }
+    if (!use_small) {
+        // child-ordered layout: slots of the edges, and which slot every node's bf16 row goes to; S starts at zero
+        JDB_CUDA_TRY(cudaMemsetAsync(w.slot_of_pos, 0xFF, w.slot_of_pos_bytes, st));
+        JDB_CUDA_TRY(cudaMemsetAsync(w.S, 0, w.s_bytes, st));
+        edge_count_kernel<<<w.n_scan_blocks, SCAN_TB, 0, st>>>(a, w.block_sum);
+        edge_scan_kernel<<<1, SCAN_TB, 0, st>>>(a, w.block_sum, w.n_scan_blocks);
+        const long long want = ((long long)ni + 1 + 7) / 8;
+        edge_fill_kernel<<<(int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16), 256, 0, st>>>(a, w.block_sum);
+        JDB_CUDA_TRY(cudaGetLastError());
     }
     if ((ls = launch(EPI_XPROJ, tmX, tmW, tmWl, (long long)N + 2 * BM, 0, 256, 4 * Hp, kd)) != JDB_OK) return ls;
     if (fa.ev_xproj_done) JDB_CUDA_TRY(cudaEventRecord(fa.ev_xproj_done, st));
-    // levels [1, last_own] run as launches of their own: all of them without the cooperative kernel, the leading
-    // wide ones with it
-    int last_own = n_levels - 1;
-    if (use_small) last_own = (n_levels >= 0 && n_wide > n_levels - 1) ? n_levels - 1 : n_wide;  // n_wide is 0 when the counts are unknown
-    if (last_own < 0) last_own = 0;
-    if (last_own >= 1) {
-        if ((ls = launch(EPI_G, tmHB, tmUf, tmUf, N, 0, bng, Hp, kh)) != JDB_OK) return ls;
+    if (!use_small) {
         const int cs_blocks = (int)((ni + 7) / 8 < (size_t)n_sm * 8 ? (ni + 7) / 8 : (size_t)n_sm * 8);
-        for (int level = 1; level <= last_own; ++level) {
-            JDB_CUDA_TRY(launch_behind(gather_kernel, dim3(cs_blocks), dim3(256), 0, st, a, level));
+        for (int level = 1; level < n_levels; ++level) {
+            JDB_CUDA_TRY(launch_behind(tune.pdl, childsum_kernel, dim3(cs_blocks), dim3(256), 0, st, a, level));
+            if ((ls = launch(EPI_F, tmHB, tmUf, tmUf, (long long)fa.n_edges, level, bnf, Hp, kh)) != JDB_OK) return ls;
             if ((ls = launch(EPI_LEVEL, tmHS, tmUiou, tmUiou, (long long)ni, level, 192, 3 * Hp, kh)) != JDB_OK) return ls;
-            if (level < last_own)   // the cooperative kernel computes its forget gates from h itself
-                if ((ls = launch(EPI_G, tmHB, tmUf, tmUf, (long long)ni, level, bng, Hp, kh)) != JDB_OK) return ls;
         }
         JDB_CUDA_TRY(cudaGetLastError());
-    }
-    if (use_small && (n_levels < 0 || last_own + 1 < n_levels)) {
-        jdb_status s = small_levels_enqueue(fa, packed_tc, P, hb, inv, n_internal_bound, last_own + 1, timeout_ns, st);
+    } else {
+        jdb_status s = small_levels_enqueue(fa, packed_tc, w.P, w.hb, w.inv, n_internal_bound, 1, timeout_ns, st);
         if (s != JDB_OK) return s;
     }
     if (fa.ev_levels_done) JDB_CUDA_TRY(cudaEventRecord(fa.ev_levels_done, st));

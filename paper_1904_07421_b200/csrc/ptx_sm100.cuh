@@ -71,22 +71,16 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
-// The same wait for a converged warp in which ONE lane consumes what the barrier guards (the lane that issues the
-// tensor-core instructions): that lane polls, so the thread that observed the phase is the thread that acts on it,
-// and the others get the result by shuffle.  Thirty-two lanes polling one barrier would be thirty-two serialised
-// shared-memory operations per poll.
-__device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, volatile int* abort, bool me, int src_lane,
-                                               unsigned long long timeout_ns = 2000000000ull) {
-    int ok = 1;
-    if (me) ok = mbar_wait(bar, parity, abort, timeout_ns) ? 1 : 0;
-    ok = __shfl_sync(0xffffffffu, ok, src_lane);
-    __syncwarp();  // memory ordering among the lanes: what the polling lane acquired is visible to the others
-    return ok != 0;
-}
-// Lane 0 polls for a warp whose lanes all use what the barrier guards only after a warp-wide barrier of their own.
+// The same wait for a converged warp whose lanes all use what the barrier guards only after a warp-wide barrier of
+// their own: lane 0 polls (thirty-two lanes polling one barrier would be thirty-two serialised shared-memory
+// operations per poll) and the others receive its verdict by shuffle, so the result is uniform over the warp.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort,
                                                unsigned long long timeout_ns = 2000000000ull) {
-    return mbar_wait_lane(bar, parity, abort, (threadIdx.x & 31) == 0, 0, timeout_ns);
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort, timeout_ns) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();  // memory ordering among the lanes: what the polling lane acquired is visible to the others
+    return ok != 0;
 }
 
 // ---- programmatic dependent launch ------------------------------------------------------------------
@@ -120,12 +114,25 @@ __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
 }
 
 // ---- tcgen05 --------------------------------------------------------------------------------------
+// TMEM allocation.  Every tcgen05 instruction of a kernel names the same CTA group: a kernel of lone CTAs uses the
+// cta_group::1 forms, a kernel of CTA pairs the cta_group::2 forms, which one warp of EACH CTA of the pair executes
+// together (both CTAs receive the same column range).
+template <int GROUP = 1>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {  // whole warp
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (GROUP == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
 }
+template <int GROUP = 1>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  // whole warp
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    if (GROUP == 2)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }

@@ -26,6 +26,21 @@ enum { BAR_MAIN = 1, BAR_META = 2 };
 __device__ __forceinline__ void named_bar(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
+// The same barrier carrying a vote: returns true in EVERY participating thread if any of them passed true.
+// Whether to leave a loop is decided through this, never by each thread reading a flag that another role of the
+// CTA may be writing at that moment: a split decision would leave some threads waiting at the next barrier.
+__device__ __forceinline__ bool named_bar_any(int id, int threads, bool mine) {
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %3, 0;\n\t"
+        "bar.red.or.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"(id), "r"(threads), "r"((uint32_t)mine)
+        : "memory");
+    return any != 0;
+}
 
 // What the arithmetic warps need to know about one pass; written by the description warps.
 struct PassSlot {
@@ -124,9 +139,9 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
             const int ne = R.t_wsum[0] + R.t_wsum[1];
             for (int et0 = 0; et0 < ne && alive; et0 += et, ++k) {
                 const int s = k & 1;
-                if (!ptx::mbar_wait_warp(ptx::smem_u32(&R.bar_empty[s]), (uint32_t)(((k >> 1) & 1) ^ 1), abort)) *abort = 1;
-                named_bar(BAR_META, META_THREADS);
-                if (*abort) { alive = false; break; }
+                const bool got = ptx::mbar_wait_warp(ptx::smem_u32(&R.bar_empty[s]), (uint32_t)(((k >> 1) & 1) ^ 1), abort);
+                if (!got) *abort = 1;
+                if (named_bar_any(BAR_META, META_THREADS, !got || *abort != 0)) { alive = false; break; }  // one verdict for all four warps
                 PassSlot& S = R.slot[s];
                 if (tm < NT_MAX) {
                     S.nodes[tm] = v;
@@ -167,8 +182,9 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
 // Grid barrier among the arithmetic warps of the participating CTAs (all of them arrive; thread 0 waits).
 // `target` = barriers passed so far + 1, times the number of participating CTAs, on the monotonically increasing
 // counter meta[META_BARRIER].  Bounded by timeout_ns; on expiry the timeout word is raised (which releases every
-// other waiter) and *abort is set.  Returns with all MAIN_THREADS threads synchronised.
-__device__ __forceinline__ void main_grid_barrier(int32_t* meta, unsigned target, unsigned long long timeout_ns,
+// other waiter) and *abort is set.  Returns with all MAIN_THREADS threads synchronised, and the same verdict in all
+// of them: false when the wait was given up here or *abort was seen raised by anybody.
+__device__ __forceinline__ bool main_grid_barrier(int32_t* meta, unsigned target, unsigned long long timeout_ns,
                                                   volatile int* abort, int tid) {
     named_bar(BAR_MAIN, MAIN_THREADS);  // every store of the arithmetic warps is ordered before the release below
     if (tid == 0) {
@@ -189,7 +205,7 @@ __device__ __forceinline__ void main_grid_barrier(int32_t* meta, unsigned target
             }
         }
     }
-    named_bar(BAR_MAIN, MAIN_THREADS);
+    return !named_bar_any(BAR_MAIN, MAIN_THREADS, *abort != 0);
 }
 
 }  // namespace small

@@ -16,16 +16,18 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libjdb.so")
 
-OK, ERR_INVALID_ARG, ERR_NOT_A_FOREST, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = range(7)
+OK, ERR_INVALID_ARG, ERR_NOT_A_FOREST, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_CHECK = range(8)
 FP32, BF16 = 0, 1
-FLAG_NO_SYNC = 1
+FLAG_NO_SYNC, FLAG_DEBUG_CHECKS = 1, 2
+TUNE_SET, TUNE_PAIR_XPROJ, TUNE_PAIR_LEVEL, TUNE_PAIR_FORGET, TUNE_TWO_ISSUERS, TUNE_NO_PDL, TUNE_PLAIN_STORES = 1, 2, 4, 8, 16, 32, 64
 MODE_AUTO, MODE_PER_LEVEL, MODE_PERSISTENT = 0, 1, 2
 META_INTS = 16
 
 EXPORTS = [
     "jdb_status_string", "jdb_last_cuda_error", "jdb_schedule_workspace_bytes", "jdb_schedule",
     "jdb_schedule_async", "jdb_schedule_static", "jdb_packed_weights_bytes", "jdb_pack_weights", "jdb_forward_workspace_bytes",
-    "jdb_treelstm_forward", "jdb_sched_status", "jdb_forward_host_workspace_bytes", "jdb_treelstm_forward_host",
+    "jdb_treelstm_forward", "jdb_sched_status", "jdb_debug_report", "jdb_forward_host_workspace_bytes",
+    "jdb_treelstm_forward_host",
 ]
 
 
@@ -39,7 +41,7 @@ class CSched(C.Structure):
 
 
 class COpts(C.Structure):
-    _fields_ = [("precision", C.c_int32), ("mode", C.c_int32), ("flags", C.c_int32), ("reserved1", C.c_int32),
+    _fields_ = [("precision", C.c_int32), ("mode", C.c_int32), ("flags", C.c_int32), ("tuning", C.c_int32),
                 ("barrier_timeout_ns", C.c_uint64), ("ev_begin", C.c_void_p), ("ev_xproj_done", C.c_void_p),
                 ("ev_levels_done", C.c_void_p), ("trace", C.c_void_p), ("trace_cap", C.c_int64)]
 
@@ -87,6 +89,8 @@ def lib():
                                        C.POINTER(COpts), vp, sz, vp]
     L.jdb_sched_status.restype = C.c_int
     L.jdb_sched_status.argtypes = [C.POINTER(CSched), C.POINTER(i32), C.POINTER(i32), vp]
+    L.jdb_debug_report.restype = C.c_int
+    L.jdb_debug_report.argtypes = [C.POINTER(CSched), C.POINTER(i32 * 4), vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
     L.jdb_forward_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
     L.jdb_treelstm_forward_host.restype = C.c_int
@@ -209,7 +213,7 @@ def jdb_treelstm_forward(forest: Forest, sched: Schedule, x: torch.Tensor, packe
                          precision: int, mode: int = MODE_AUTO, h: Optional[torch.Tensor] = None,
                          c: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None,
                          barrier_timeout_ns: int = 0, prof_events=None,
-                         trace: Optional[torch.Tensor] = None):
+                         trace: Optional[torch.Tensor] = None, flags: int = 0, tuning: int = 0):
     """h, c [n_nodes, H] fp32 of every node; x is fp32 or bfloat16 [n_nodes, >= D] with row stride x.stride(0)."""
     dev = forest.child_ptr.device
     n = forest.n_nodes
@@ -226,7 +230,7 @@ def jdb_treelstm_forward(forest: Forest, sched: Schedule, x: torch.Tensor, packe
     assert x.stride(1) == 1 and h.stride(1) == 1 and c.stride(1) == 1 and h.stride(0) == c.stride(0)
     ws = forward_workspace(forest, sched, D, H, precision) if ws is None else ws
     cf, cs = forest.c(), sched.c()
-    opts = COpts(precision, mode, 0, 0, barrier_timeout_ns)
+    opts = COpts(precision, mode, flags, tuning, barrier_timeout_ns)
     if prof_events is not None:  # three torch.cuda.Event(enable_timing=True): begin, projection done, levels done
         for ev in prof_events:
             if ev.cuda_event == 0:
@@ -249,6 +253,16 @@ def jdb_sched_status(sched: Schedule, stream=None):
     if st != OK:
         raise JdbError(st, "jdb_sched_status")
     return nl.value, nv.value
+
+
+def jdb_debug_report(sched: Schedule, stream=None):
+    """(check, value, bound, where) recorded by a forward run with FLAG_DEBUG_CHECKS; check 0 means none failed."""
+    cs = sched.c()
+    out = (C.c_int32 * 4)()
+    st = lib().jdb_debug_report(C.byref(cs), C.byref(out), _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_debug_report")
+    return tuple(out)
 
 
 class StepPlan:
@@ -306,13 +320,13 @@ def forward_host_workspace(n_nodes: int, n_edges: int, D: int, H: int, precision
 
 def jdb_treelstm_forward_host(child_ptr: torch.Tensor, child_idx: torch.Tensor, x: torch.Tensor, packed: torch.Tensor,
                               D: int, H: int, precision: int, h: torch.Tensor, c: torch.Tensor, dev_ws: torch.Tensor,
-                              stream=None) -> int:
+                              stream=None, flags: int = 0) -> int:
     """Host tensors in (CSR int32, x dense), host tensors out (h, c dense fp32).  Returns n_levels."""
     n, e = int(child_ptr.numel() - 1), int(child_idx.numel())
     for t in (child_ptr, child_idx, x, h, c):
         assert not t.is_cuda and t.is_contiguous()
     x_dtype = BF16 if x.dtype == torch.bfloat16 else FP32
-    opts = COpts(precision, MODE_AUTO, 0, 0, 0, None, None, None, None, 0)
+    opts = COpts(precision, MODE_AUTO, flags, 0, 0, None, None, None, None, 0)
     nl = C.c_int32(0)
     st = lib().jdb_treelstm_forward_host(_ptr(child_ptr), _ptr(child_idx), n, e, _ptr(x), x_dtype, _ptr(packed), D, H,
                                          _ptr(h), _ptr(c), C.byref(opts), _ptr(dev_ws), dev_ws.numel(), C.byref(nl),

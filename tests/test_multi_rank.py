@@ -46,3 +46,24 @@ def test_rank_zero_matches_the_single_gpu_workload():
     from paper_1904_07421_b200 import workloads as wl
     a, b = bench.rank_workload(2, 0), wl.make_workload(2)
     assert np.array_equal(a.forest.child_idx, b.forest.child_idx) and np.array_equal(a.token, b.token)
+
+
+def test_bench_starts_its_own_ranks_when_launched_bare():
+    """`python bench.py --gpus 2` without WORLD_SIZE re-launches itself as two ranks on 127.0.0.1; with
+    --rendezvous-only the ranks meet over gloo on the CPU, reduce the totals like the timed path does, and rank 0
+    prints one line that says n_gpus = 2."""
+    import json
+    import subprocess
+    import bench
+    cmd = bench.launcher_command(2, ["--gpus", "2", "--rendezvous-only"], 29400)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rendezvous-only"],
+                         capture_output=True, text=True, timeout=240, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    n0 = bench.rank_workload(1, 0).forest.n_nodes
+    n1 = bench.rank_workload(1, 1).forest.n_nodes
+    assert out["n_gpus"] == 2 and out["max_seconds"] == 2.0 and out["total_nodes"] == float(n0 + n1)

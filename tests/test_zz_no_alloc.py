@@ -43,6 +43,13 @@ def test_static_scratch_schedule_matches_the_workspace_one_twice():
     assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
     _compare(f1, out1, ref1)
     _compare(f2, out2, ref2)
+    # and directly against the CPU checker, so that this entry point does not lean on the other one being right
+    from oracle import schedule as osched
+    for forest_np, out in ((w1.forest, out1), (w2, out2)):
+        depth, level_ptr, perm, _, n_levels = osched.schedule(forest_np.child_ptr, forest_np.child_idx, forest_np.n_nodes)
+        assert out.n_levels == n_levels
+        assert np.array_equal(out.depth.cpu().numpy(), depth) and np.array_equal(out.perm.cpu().numpy(), perm)
+        assert np.array_equal(out.level_ptr[:n_levels + 1].cpu().numpy(), level_ptr)
 
 
 def test_static_scratch_schedule_limits_and_errors():
