@@ -154,6 +154,25 @@ jdb_status jdb_schedule_async(const jdb_forest *forest, jdb_sched *out, void *ws
 #define JDB_STATIC_MAX_NODES 65536
 jdb_status jdb_schedule_static(const jdb_forest *forest, jdb_sched *out, void *stream);
 
+/* ---- launch counts at two granularities (Section 3: kernel versus subgraph statistics) ------- */
+
+/* How many launches the forest costs without and with batching, counted at cell (subgraph) granularity, where two
+ * cells share a launch only if they agree in depth and in their number of children, and at operator (kernel)
+ * granularity, where 29 of a cell's 33 operators are shared by all cells of a depth and the 4 that depend on the
+ * number of children are shared per (depth, number of children):
+ *     cells:      n_nodes                 ->  number of distinct (depth, children) pairs
+ *     operators:  33 * n_nodes            ->  sum over depths of (29 + 4 * kinds of cell at that depth)
+ * The ratio unbatched / batched of a column is that granularity's batching ratio.  `sched` must come from
+ * jdb_schedule on `forest`; `out` is a HOST struct; `ws` is device scratch of jdb_launch_counts_workspace_bytes
+ * bytes, 8-byte aligned.  Synchronises `stream` once. */
+typedef struct {
+    int64_t cells_unbatched, cells_batched, ops_unbatched, ops_batched;
+    int32_t n_levels, reserved;
+} jdb_launch_stats;
+size_t jdb_launch_counts_workspace_bytes(int32_t n_nodes);
+jdb_status jdb_launch_counts(const jdb_forest *forest, const jdb_sched *sched, jdb_launch_stats *out, void *ws,
+                             size_t ws_bytes, void *stream);
+
 /* ---- batched execution (Section 4.3: stack, run the common subgraph once, slice) ------------ */
 
 /* Weights arrive as the cell's natural matrices: W [4H, D], U [4H, H], b [4H], fp32 row-major, gate

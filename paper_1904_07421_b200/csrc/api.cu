@@ -300,7 +300,10 @@ jdb_status jdb_treelstm_forward_host(const int32_t* child_ptr, const int32_t* ch
     if (n_edges > 0) JDB_CUDA_TRY(cudaMemcpyAsync(d_ci, child_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice, st));
     JDB_CUDA_TRY(cudaMemcpyAsync(d_x, x, n * (size_t)D * xb, cudaMemcpyHostToDevice, st));
     jdb_forest f{d_cp, d_ci, n_nodes, n_edges};
-    jdb_status s = jdb_schedule_async(&f, &sch, d_sws, sws, stream);
+    // per-level launches (tensor-core path beyond the cooperative kernel's hidden sizes) need the level count on the
+    // host: there the analysis synchronises, and the forward is sized by the real number of internal nodes
+    const bool per_level = opts->precision == JDB_BF16 && !small_levels_supported(H);
+    jdb_status s = per_level ? jdb_schedule(&f, &sch, d_sws, sws, stream) : jdb_schedule_async(&f, &sch, d_sws, sws, stream);
     if (s != JDB_OK) return s;
     // enqueue the forward and the copies back before the one synchronisation
     jdb_opts o = *opts;

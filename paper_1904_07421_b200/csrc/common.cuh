@@ -48,6 +48,33 @@ struct DevInfo {
 enum { ATTR_SMALL_SCHED = 1, ATTR_GEMM_TC = 2, ATTR_SMALL_LEVELS = 4, ATTR_SMALL_F32 = 8 };
 DevInfo* dev_info();  // of the current device; nullptr if the runtime fails
 
+// JDB_FLAG_DEBUG_CHECKS: true if 0 <= v < bound.  Otherwise the first offender of the call is recorded in meta
+// (what, value, bound, where) and the caller skips the access.
+enum { CHECK_PERM = 1, CHECK_CHILD = 2, CHECK_POSITION = 3, CHECK_SLOT = 4, CHECK_PARENT_ROW = 5, CHECK_LEVEL_PTR = 6,
+       CHECK_EDGE_PTR = 7 };
+#ifdef __CUDACC__
+__device__ __forceinline__ bool dbg_ok(int32_t* meta, int what, long long v, long long bound, int where) {
+    if (v >= 0 && v < bound) return true;
+    if (atomicCAS(&meta[META_CHECK], 0, what) == 0) {
+        meta[META_CHECK + 1] = (int32_t)(v < -2147483647LL ? -2147483647LL : (v > 2147483647LL ? 2147483647LL : v));
+        meta[META_CHECK + 2] = (int32_t)(bound > 2147483647LL ? 2147483647LL : bound);
+        meta[META_CHECK + 3] = where;
+    }
+    return false;
+}
+// Positions [lo, hi) of a level; with debug checks an inconsistent pair is recorded and the level made empty (every
+// reader of the same pair takes the same decision).
+__device__ __forceinline__ void checked_level(const int32_t* level_ptr, int level, int n_nodes, int32_t* meta, int debug,
+                                              int& lo, int& hi) {
+    lo = level_ptr[level];
+    hi = level_ptr[level + 1];
+    if (debug && !(dbg_ok(meta, CHECK_LEVEL_PTR, lo, (long long)n_nodes + 1, level) &&
+                   dbg_ok(meta, CHECK_LEVEL_PTR, hi, (long long)n_nodes + 1, level) &&
+                   dbg_ok(meta, CHECK_LEVEL_PTR, hi - lo, (long long)n_nodes + 1, level)))
+        lo = hi = 0;
+}
+#endif
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 

@@ -39,7 +39,11 @@ __global__ void __launch_bounds__(512) xproj_simt_kernel(ForwardArgs a, int jt, 
     const int n_leaves = a.meta[META_N_LEAVES];
     const int pos0 = blockIdx.x * TM;
     const int tx = threadIdx.x % jt, ky = threadIdx.x / jt;
-    if (threadIdx.x < TM) nodes[threadIdx.x] = (pos0 + threadIdx.x < N) ? a.perm[pos0 + threadIdx.x] : -1;
+    if (threadIdx.x < TM) {
+        int v = (pos0 + threadIdx.x < N) ? a.perm[pos0 + threadIdx.x] : -1;
+        if (a.debug && v != -1 && !dbg_ok(a.meta, CHECK_PERM, v, N, pos0 + threadIdx.x)) v = -1;
+        nodes[threadIdx.x] = v;
+    }
     __syncthreads();
     for (int idx = threadIdx.x; idx < TM * D; idx += blockDim.x) {
         int t = idx / D, d = idx - t * D;
@@ -120,9 +124,14 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
 
     if (tid < TM) {
         int v = tid < m ? a.perm[pos0 + tid] : -1;
+        if (a.debug && v != -1 && !dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, pos0 + tid)) v = -1;
         nodes[tid] = v;
-        ebeg[tid] = v >= 0 ? a.child_ptr[v] : 0;
-        eoff[tid + 1] = v >= 0 ? a.child_ptr[v + 1] - a.child_ptr[v] : 0;
+        int eb = v >= 0 ? a.child_ptr[v] : 0, cnt = v >= 0 ? a.child_ptr[v + 1] - eb : 0;
+        if (a.debug && !(dbg_ok(a.meta, CHECK_EDGE_PTR, eb, (long long)a.n_edges + 1, pos0 + tid) &&
+                         dbg_ok(a.meta, CHECK_EDGE_PTR, cnt, (long long)a.n_edges - eb + 1, pos0 + tid)))
+            eb = cnt = 0;
+        ebeg[tid] = eb;
+        eoff[tid + 1] = cnt;
     }
     __syncthreads();
     if (tid == 0) {
@@ -137,7 +146,11 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
         float s = 0.f;
         if (t < m && jj < H) {
             const int e0 = ebeg[t], e1 = e0 + (eoff[t + 1] - eoff[t]);
-            for (int e = e0; e < e1; ++e) s += __ldcg(&a.h[(int64_t)a.child_idx[e] * a.ldh + jj]);
+            for (int e = e0; e < e1; ++e) {
+                const int k = a.child_idx[e];
+                if (a.debug && !dbg_ok(a.meta, CHECK_CHILD, k, a.n_nodes, e)) continue;
+                s += __ldcg(&a.h[(int64_t)k * a.ldh + jj]);
+            }
             if (a.round_bf16) s = bf16r(s);
         }
         hs[idx] = s;
@@ -200,6 +213,7 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
                 const int e = e0 + tid;
                 while (eoff[t + 1] <= e) ++t;
                 k = a.child_idx[ebeg[t] + (e - eoff[t])];
+                if (a.debug && !dbg_ok(a.meta, CHECK_CHILD, k, a.n_nodes, ebeg[t] + (e - eoff[t]))) k = -1;
             }
             ck_t[tid] = t;
             ck_k[tid] = k;
@@ -208,7 +222,7 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
         for (int idx = tid; idx < TE * Hs; idx += nt) {
             const int ee = idx / Hs, jj = idx - ee * Hs;
             float val = 0.f;
-            if (ee < nc && jj < H) {
+            if (ee < nc && jj < H && ck_k[ee] >= 0) {
                 val = __ldcg(&a.h[(int64_t)ck_k[ee] * a.ldh + jj]);
                 if (a.round_bf16) val = bf16r(val);
             }
@@ -241,7 +255,7 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
                 }
 #pragma unroll
                 for (int ee = 0; ee < TE; ++ee) {
-                    if (ee < nc) {
+                    if (ee < nc && ck_k[ee] >= 0) {
                         const int t = ck_t[ee];
                         const float f = sigmoid_acc(pf[t * Hs + j] + dot[ee]);
                         cacc[t * Hs + j] = fmaf(f, __ldcg(&a.c[(int64_t)ck_k[ee] * a.ldh + j]), cacc[t * Hs + j]);
@@ -255,6 +269,7 @@ __device__ void level_tile(const ForwardArgs& a, int pos0, int m, int n_leaves, 
     // h = o * tanh(c); rows back to node order
     for (int idx = tid; idx < m * H; idx += nt) {
         const int t = idx / H, j = idx - t * H;
+        if (nodes[t] < 0) continue;
         const int64_t row = (int64_t)nodes[t] * a.ldh;
         const float cc = cacc[t * Hs + j];
         a.c[row + j] = cc;
@@ -267,7 +282,9 @@ __global__ void __launch_bounds__(512) level_kernel(ForwardArgs a, int level, in
     extern __shared__ float sm[];
     const int n_levels = a.meta[META_N_LEVELS];
     if (level >= n_levels) return;
-    const int lo = a.level_ptr[level], hi = a.level_ptr[level + 1], n_leaves = a.level_ptr[1];
+    const int n_leaves = a.level_ptr[1];
+    int lo, hi;
+    checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
     const int tiles = (hi - lo + TM - 1) / TM;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x)
         level_tile(a, lo + tile * TM, min(TM, hi - lo - tile * TM), n_leaves, sm, jt, ks);
@@ -279,7 +296,8 @@ __global__ void __launch_bounds__(512) persistent_kernel(ForwardArgs a, unsigned
     if (a.meta[META_ERROR] != 0 || a.meta[META_UNFINISHED] != 0) return;  // malformed forest: nothing to run
     const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
     for (int level = 1; level < n_levels; ++level) {
-        const int lo = a.level_ptr[level], hi = a.level_ptr[level + 1];
+        int lo, hi;
+        checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
         const int tiles = (hi - lo + TM - 1) / TM;
         for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x)
             level_tile(a, lo + tile * TM, min(TM, hi - lo - tile * TM), n_leaves, sm, jt, ks);

@@ -64,6 +64,7 @@ struct SmallArgs {
     unsigned long long timeout_ns;
     int32_t first_level;  // levels below it were evaluated by launches of their own
     int32_t n_nodes, n_edges;
+    int32_t debug;        // check every index against its array before following it
     unsigned long long* trace;
     long long trace_cap;
 };
@@ -127,7 +128,9 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
     {
         int mt = 1;
         for (int l = a.first_level + tid; l < n_levels; l += STHREADS) {
-            const int ln = a.level_ptr[l + 1] - a.level_ptr[l], nt = tile_nodes(ln, nt_max, n_grp);
+            int llo, lhi;
+            checked_level(a.level_ptr, l, a.n_nodes, a.meta, a.debug, llo, lhi);
+            const int ln = lhi - llo, nt = tile_nodes(ln, nt_max, n_grp);
             mt = max(mt, (ln + nt - 1) / nt);
         }
         if (mt > 1) atomicMax(&s_max_tiles, mt);
@@ -140,7 +143,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
     if (warp >= MAIN_WARPS) {
         // ================= description warps: run ahead of the arithmetic by up to two passes =================
         if (alive) {
-            DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, a.inv, a.first_level, n_levels, grp, n_grp, active_grp, nt_max};
+            DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, a.inv, a.first_level, n_levels, grp, n_grp, active_grp, nt_max,
+                           a.meta, a.n_nodes, a.n_edges, a.debug};
             describe_passes(d, ring, ET, abort, tid - MAIN_THREADS, [&](int pos0, int m, int tcount, int tm) {
                 // forget slices of the tile's input projection, for this CTA's hidden units (parity selects the buffer)
                 float* dst = pfs + (tcount & 1) * (NT_MAX * PF_LD);
@@ -163,7 +167,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
         uint32_t mma_phase = 0;
         int k = 0, tcount = 0;
         for (int level = a.first_level; level < n_levels && alive; ++level) {
-            const int lo = a.level_ptr[level], hi = a.level_ptr[level + 1];
+            int lo, hi;
+            checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
             const int nt = tile_nodes(hi - lo, nt_max, n_grp);
             const int tiles = (hi - lo + nt - 1) / nt;
             stamp(level, 0, true);
@@ -277,6 +282,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                             const float cc = fmaf(sigmoid_fast(zi[i] + pi[i]), tanh_fast(zu[i] + pu[i]), sfc[i]);
                             const float hh = sigmoid_fast(zo[i] + po[i]) * tanh_fast(cc);
                             const int vnode = S.nodes[r];
+                            if (vnode < 0) continue;  // a row whose node id failed the debug checks
                             if (j0 + lane < H) {
                                 a.c[(int64_t)vnode * a.ldh + j0 + lane] = cc;
                                 a.h[(int64_t)vnode * a.ldh + j0 + lane] = hh;
@@ -348,6 +354,7 @@ jdb_status small_levels_enqueue(const ForwardArgs& fa, const void* packed_tc, co
     a.trace_cap = fa.trace_cap;
 
     a.n_nodes = fa.n_nodes; a.n_edges = fa.n_edges;
+    a.debug = fa.debug;
     int groups = n_sm / a.n_slices;  // one CTA per SM: the kernel uses most of an SM's shared memory
     const int max_tiles = ceil_div(n_internal_bound > 0 ? n_internal_bound : 1, 32);
     if (groups > max_tiles) groups = max_tiles;

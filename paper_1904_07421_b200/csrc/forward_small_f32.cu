@@ -48,6 +48,8 @@ struct F32Args {
     const int32_t* perm;
     int32_t* meta;
     int32_t H, n_slices;
+    int32_t n_nodes, n_edges;
+    int32_t debug;       // check every index against its array before following it
     const float4* Ut4;   // [H][H]: Ut4[k * H + j] = (U_i, U_o, U_u, U_f)[j][k]
     const float4* P4;    // [n_internal][H]: biased input projection (i, o, u, f), rows in level order
     float* h;
@@ -109,7 +111,9 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
     {
         int mt = 1;
         for (int l = 1 + tid; l < n_levels; l += STHREADS) {
-            const int ln = a.level_ptr[l + 1] - a.level_ptr[l], nt = tile_nodes(ln, FNT_RULE, n_grp);
+            int llo, lhi;
+            checked_level(a.level_ptr, l, a.n_nodes, a.meta, a.debug, llo, lhi);
+            const int ln = lhi - llo, nt = tile_nodes(ln, FNT_RULE, n_grp);
             mt = max(mt, (ln + nt - 1) / nt);
         }
         if (mt > 1) atomicMax(&s_max_tiles, mt);
@@ -122,7 +126,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
     if (warp >= MAIN_WARPS) {
         // ================= description warps =================
         if (alive) {
-            DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, nullptr, 1, n_levels, grp, n_grp, active_grp, FNT_RULE};
+            DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, nullptr, 1, n_levels, grp, n_grp, active_grp, FNT_RULE,
+                           a.meta, a.n_nodes, a.n_edges, a.debug};
             describe_passes(d, ring, FET, abort, tid - MAIN_THREADS, [&](int pos0, int m, int tcount, int tm) {
                 // the tile's input projection for this CTA's hidden units (parity selects the buffer)
                 float4* dst = pst + (tcount & 1) * (FNT * SBJ);
@@ -147,7 +152,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
         const float4* hk4 = reinterpret_cast<const float4*>(hk);
         int k = 0, tcount = 0;
         for (int level = 1; level < n_levels && alive; ++level) {
-            const int lo = a.level_ptr[level], hi = a.level_ptr[level + 1];
+            int lo, hi;
+            checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
             const int nt = tile_nodes(hi - lo, FNT_RULE, n_grp);
             const int tiles = (hi - lo + nt - 1) / nt;
             stamp(level, 0, true);
@@ -240,7 +246,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
                             zu[i] += src[2 * SBJ];
                             sfc[i] += src[3 * SBJ];
                         }
-                        if (last && j0 + lane < H) {
+                        if (last && j0 + lane < H && S.nodes[r] >= 0) {
                             const float4 p = pst[(tcount & 1) * (FNT * SBJ) + r * SBJ + lane];
                             const float cc = fmaf(sigmoid_acc(zi[i] + p.x), tanhf(zu[i] + p.z), sfc[i]);
                             const int64_t row = (int64_t)S.nodes[r] * a.ldh;
@@ -285,6 +291,7 @@ jdb_status small_levels_f32_enqueue(const ForwardArgs& fa, int n_internal_bound,
     F32Args a{};
     a.child_ptr = fa.child_ptr; a.child_idx = fa.child_idx; a.level_ptr = fa.level_ptr; a.perm = fa.perm;
     a.meta = fa.meta; a.H = H;
+    a.n_nodes = fa.n_nodes; a.n_edges = fa.n_edges; a.debug = fa.debug;
     a.n_slices = (H + SBJ - 1) / SBJ;
     a.Ut4 = (const float4*)fa.Ut;
     a.P4 = (const float4*)fa.P;

@@ -41,6 +41,11 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES_MAX = MAX_BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES_MAX;
 constexpr int GEMM1_THREADS = 224;  // warp 0: TMA producer, warps 1 and 6: MMA issuers, warps 2-5: epilogue
+// The forget-gate GEMM's epilogue is instruction-bound (a segmented sum over the accumulator rows per 16-column
+// step), and a scheduler with a single warp issues well below one instruction per cycle: it runs EIGHT epilogue
+// warps, two per TMEM lane quarter and per scheduler, which take the steps of a tile alternately.
+constexpr int GEMMF_THREADS = 320;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
+__host__ __device__ constexpr int gemm_threads(int epi) { return epi == 2 ? GEMMF_THREADS : GEMM1_THREADS; }
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;
 constexpr int TMEM_COLS = 512;  // two accumulator buffers of up to 256 columns
 
@@ -75,20 +80,6 @@ struct TcArgs {
     int32_t* slot_child;  // [n_edges]         node id of the child at the slot
     int32_t debug;        // check every index against its array before following it
 };
-
-// JDB_FLAG_DEBUG_CHECKS: true if 0 <= v < bound.  Otherwise the first offender of the call is recorded in meta
-// (what, value, bound, where) and the caller skips the access.
-enum { CHECK_PERM = 1, CHECK_CHILD = 2, CHECK_POSITION = 3, CHECK_SLOT = 4, CHECK_PARENT_ROW = 5, CHECK_LEVEL_PTR = 6,
-       CHECK_EDGE_PTR = 7 };
-__device__ __forceinline__ bool dbg_ok(int32_t* meta, int what, long long v, long long bound, int where) {
-    if (v >= 0 && v < bound) return true;
-    if (atomicCAS(&meta[META_CHECK], 0, what) == 0) {
-        meta[META_CHECK + 1] = (int32_t)(v < -2147483647LL ? -2147483647LL : (v > 2147483647LL ? 2147483647LL : v));
-        meta[META_CHECK + 2] = (int32_t)(bound > 2147483647LL ? 2147483647LL : bound);
-        meta[META_CHECK + 3] = where;
-    }
-    return false;
-}
 
 // Where a tile sits.  The input projection walks the rows in level order and never mixes
 // leaves and internal nodes in a tile: leaf tiles need only the i, o, u blocks (192 of the 256 columns of a
@@ -135,7 +126,9 @@ constexpr int GEMM_SMEM_STORE = GEMM_SMEM + 4 * EPI_STEP_FLOATS * 4;   // input 
 // arrays (the parent's forget pre-activation and the child's c)
 constexpr int F_STEP_FLOATS = 2 * 32 * 16;
 constexpr int F_STAGES = 3;
-constexpr int F_SCRATCH_BYTES = 4 * EPI_RING * F_STEP_FLOATS * 4;
+constexpr int F_RING = 2;   // this step's buffer and the next one's (of the warp's own steps, which are every other step)
+constexpr int F_WARPS = 8;
+constexpr int F_SCRATCH_BYTES = F_WARPS * F_RING * F_STEP_FLOATS * 4;
 constexpr int GEMM_SMEM_F = F_STAGES * STAGE_BYTES + F_SCRATCH_BYTES + 1024;
 static_assert(GEMM_SMEM_STORE <= 227 * 1024 - 256, "GEMM shared memory");
 static_assert(GEMM_SMEM_F <= 227 * 1024 - 256, "forget GEMM shared memory");
@@ -543,8 +536,10 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         }
         cp_async_wait<0>();
     } else if (EPI == EPI_F) {
-        // rows are edge slots; the parent's forget pre-activation and the child's c arrive two steps ahead
-        float* ring = scratch + quarter * (EPI_RING * F_STEP_FLOATS);
+        // rows are edge slots; eight warps: this one takes the steps q = split, split + 2, ... of every tile, and the
+        // parent's forget pre-activation and the child's c of its next step arrive while it works on the current one
+        const int split = (warp - 2) >> 2;
+        float* ring = scratch + (warp - 2) * (F_RING * F_STEP_FLOATS);
         const uint32_t ring_addr = smem_u32(ring);
         const int steps = bn >> 4;
         auto slot_rows = [&](const Tile& ti, int (&pr)[4], int (&kd)[4]) {
@@ -561,24 +556,24 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
                 }
             }
         };
-        int f_t = t0, f_q = 0, f_buf = 0;
+        int f_t = t0, f_q = split, f_buf = 0;
         Tile f_ti = tile_at(f_t);
         int f_pr[4], f_kd[4];
         if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
         auto fetch_next = [&]() {
             if (f_t < total_tiles) {
                 forget_fetch(a, f_ti, lane, f_q, f_pr, f_kd, ring_addr + (uint32_t)f_buf * (F_STEP_FLOATS * 4), ring + f_buf * F_STEP_FLOATS);
-                if (++f_q == steps) {
-                    f_q = 0;
+                f_q += 2;
+                if (f_q >= steps) {
+                    f_q = split;
                     f_t += t_step;
                     f_ti = tile_at(f_t);
                     if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
                 }
             }
             cp_async_commit();
-            if (++f_buf == EPI_RING) f_buf = 0;
+            f_buf ^= 1;
         };
-        fetch_next();
         fetch_next();
         int cur = 0;
         for (int t = t0; t < total_tiles && ok; t += t_step) {
@@ -591,12 +586,12 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
-            for (int q = 0; q < steps; ++q) {
+            for (int q = split; q < steps; q += 2) {
+                cp_async_wait<0>();          // this step's copies have landed (they were started a step ago)
+                __syncwarp();                // ... and so have the other lanes'; the other buffer is free
                 fetch_next();
-                cp_async_wait<2>();
-                __syncwarp();
                 forget_step(a, ti, taddr, lane, q, par, runs, ring + cur * F_STEP_FLOATS);
-                if (++cur == EPI_RING) cur = 0;
+                cur ^= 1;
             }
             release_acc(acc);
             acc ^= 1;
@@ -658,12 +653,8 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
 // (forget-gate GEMM).  An inconsistent range is recorded (debug checks) and made empty.
 template <int EPI>
 __device__ __forceinline__ void level_range(const TcArgs& a, int level, int n_leaves, int& lo, int& hi) {
-    lo = a.level_ptr[level];
-    hi = a.level_ptr[level + 1];
-    bool good = !a.debug || (dbg_ok(a.meta, CHECK_LEVEL_PTR, lo, (long long)a.n_nodes + 1, level) &&
-                             dbg_ok(a.meta, CHECK_LEVEL_PTR, hi, (long long)a.n_nodes + 1, level) &&
-                             dbg_ok(a.meta, CHECK_LEVEL_PTR, hi - lo, (long long)a.n_nodes + 1, level) &&
-                             dbg_ok(a.meta, CHECK_LEVEL_PTR, lo - n_leaves, (long long)a.n_int_bound + 1, level) &&
+    checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
+    bool good = !a.debug || (dbg_ok(a.meta, CHECK_LEVEL_PTR, lo - n_leaves, (long long)a.n_int_bound + 1, level) &&
                              dbg_ok(a.meta, CHECK_LEVEL_PTR, hi - n_leaves, (long long)a.n_int_bound + 1, level));
     if (good && EPI == EPI_F) {
         lo = a.eoff[lo - n_leaves];
@@ -676,7 +667,7 @@ __device__ __forceinline__ void level_range(const TcArgs& a, int level, int n_le
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(GEMM1_THREADS, 1)
+__global__ void __launch_bounds__(gemm_threads(EPI), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
@@ -699,7 +690,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_tfull[b]), a.issuers);
-            mbar_init(smem_u32(&bar_tempty[b]), 128);
+            mbar_init(smem_u32(&bar_tempty[b]), EPI == EPI_F ? 32 * F_WARPS : 128);
         }
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -756,7 +747,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
         if (!ok && lane == 0) *abort = 1;
-    } else if (warp == 1 || (warp == 6 && a.issuers == 2)) {
+    } else if (warp == 1 || (EPI != EPI_F && warp == 6 && a.issuers == 2)) {
         // One MMA issuer for the whole tile width, or two taking half of the columns each.  The whole warp walks the pipeline (waits,
         // descriptors), so every operand of tcgen05.mma is warp-uniform; one elected lane issues.
         {
@@ -796,7 +787,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (!ok && lane == 0) *abort = 1;
         }
-    } else if (warp >= 2 && warp <= 5) {
+    } else if (warp >= 2 && warp <= (EPI == EPI_F ? 1 + F_WARPS : 5)) {
         epilogue_warps<EPI, false>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST * SB), tmem_base,
                                    bar_tfull, bar_tempty, abort, warp, lane, blockIdx.x, gridDim.x, total_tiles, n_tiles, lo, hi,
                                    bn, n_leaves, mt_leaf, 0);
@@ -827,7 +818,7 @@ constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH_BYTES + 10
 static_assert(GEMM2_SMEM_LEVEL <= 227 * 1024 - 256, "pair level GEMM shared memory");
 
 template <int EPI>
-__global__ void __launch_bounds__(GEMM1_THREADS, 1)
+__global__ void __launch_bounds__(gemm_threads(EPI), 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
@@ -868,7 +859,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_tfull[b]), 1);
-            mbar_init(smem_u32(&bar_tempty[b]), 256);  // the epilogue threads of both CTAs
+            mbar_init(smem_u32(&bar_tempty[b]), EPI == EPI_F ? 64 * F_WARPS : 256);  // the epilogue threads of both CTAs
         }
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -949,7 +940,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             if (!ok && lane == 0) *abort = 1;
         }
-    } else if (warp >= 2 && warp <= 5) {
+    } else if (warp >= 2 && warp <= (EPI == EPI_F ? 1 + F_WARPS : 5)) {
         epilogue_warps<EPI, true>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST2 * STAGE2_BYTES),
                                   tmem_base, bar_tfull, bar_tempty, abort, warp, lane, pair, n_pairs, total_tiles, n_tiles, lo, hi,
                                   bn, n_leaves, mt_leaf, (int)rank);
@@ -1434,6 +1425,8 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     };
     const int kd = L.Kd / BK, kh = Hp / BK;
 
+    TcArgs af = a;   // the forget-gate GEMM always has one MMA issuer (its warps 2-9 are all epilogue warps)
+    af.issuers = 1;
     // one GEMM launch: a lone-CTA grid, or a grid of CTA pairs (clusters of 2) for launches with many tiles
     auto launch = [&](int epi, const CUtensorMap& tA, const CUtensorMap& tB_full, const CUtensorMap& tBl, long long rows_bound,
                       int level, int bn, int n_total, int kblocks) -> jdb_status {
@@ -1446,13 +1439,13 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
             const int grid = gemm_grid(rows_bound, n_tiles);
             if (epi == EPI_XPROJ) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
             else if (epi == EPI_LEVEL) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_LEVEL>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_LEVEL, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
-            else JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_F>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_F, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+            else JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_F>, dim3(grid), dim3(GEMMF_THREADS), GEMM_SMEM_F, st, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
             return JDB_OK;
         }
         int pairs = (int)(tiles2 < n_sm / 2 ? (tiles2 > 0 ? tiles2 : 1) : n_sm / 2);
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(2 * pairs);
-        cfg.blockDim = dim3(GEMM1_THREADS);
+        cfg.blockDim = dim3(gemm_threads(epi));
         cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : epi == EPI_F ? GEMM2_SMEM_F : GEMM2_SMEM;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
@@ -1466,7 +1459,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         cfg.numAttrs = tune.pdl ? 2 : 1;
         if (epi == EPI_XPROJ) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_XPROJ>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
         else if (epi == EPI_LEVEL) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_LEVEL>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
-        else JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_F>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+        else JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_F>, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
         return JDB_OK;
     };
 

@@ -100,6 +100,8 @@ struct DescribeArgs {
     const int32_t* perm;
     const int32_t* inv;  // position of every node in level order (may be null: positions are then not filled in)
     int first_level, n_levels, grp, n_grp, active_grp, nt_max;
+    int32_t* meta;       // debug checks: where the first offending index is recorded
+    int n_nodes, n_edges, debug;
 };
 
 // The loop of the description warps (threads MAIN_THREADS .. STHREADS-1 of the CTA; tm = index among them).
@@ -115,7 +117,8 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
     int tcount = 0;  // tiles described so far
     bool alive = true;
     for (int level = d.first_level; level < d.n_levels && alive; ++level) {
-        const int lo = d.level_ptr[level], hi = d.level_ptr[level + 1];
+        int lo, hi;
+        checked_level(d.level_ptr, level, d.n_nodes, d.meta, d.debug, lo, hi);
         const int nt = tile_nodes(hi - lo, d.nt_max, d.n_grp);
         const int tiles = (hi - lo + nt - 1) / nt;
         for (int tile = d.grp; tile < tiles && alive; tile += d.active_grp, ++tcount) {
@@ -124,8 +127,12 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
             int v = -1, eb = 0, incl = 0;
             if (tm < NT_MAX) {
                 if (tm < m) v = d.perm[pos0 + tm];
+                if (d.debug && tm < m && !dbg_ok(d.meta, CHECK_PERM, v, d.n_nodes, pos0 + tm)) v = -1;  // a row without a node: no edges, nothing stored
                 int cnt = 0;
                 if (v >= 0) { eb = d.child_ptr[v]; cnt = d.child_ptr[v + 1] - eb; }
+                if (d.debug && !(dbg_ok(d.meta, CHECK_EDGE_PTR, eb, (long long)d.n_edges + 1, pos0 + tm) &&
+                                 dbg_ok(d.meta, CHECK_EDGE_PTR, cnt, (long long)d.n_edges - eb + 1, pos0 + tm)))
+                    eb = cnt = 0;
                 incl = cnt;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -165,7 +172,9 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
                         }
                         pr = lo_r;
                         kid = d.child_idx[R.t_ebeg[pr] + (e - S.eoff[pr])];
+                        if (d.debug && !dbg_ok(d.meta, CHECK_CHILD, kid, d.n_nodes, R.t_ebeg[pr] + (e - S.eoff[pr]))) kid = 0;  // reported; row 0 stands in
                         if (d.inv) kpos = d.inv[kid];
+                        if (d.debug && d.inv && !dbg_ok(d.meta, CHECK_POSITION, kpos, d.n_nodes, kid)) kpos = 0;
                     }
                     S.ek_id[tm] = kid;
                     S.ek_pos[tm] = kpos;

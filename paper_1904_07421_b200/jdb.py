@@ -27,7 +27,7 @@ EXPORTS = [
     "jdb_status_string", "jdb_last_cuda_error", "jdb_schedule_workspace_bytes", "jdb_schedule",
     "jdb_schedule_async", "jdb_schedule_static", "jdb_packed_weights_bytes", "jdb_pack_weights", "jdb_forward_workspace_bytes",
     "jdb_treelstm_forward", "jdb_sched_status", "jdb_debug_report", "jdb_forward_host_workspace_bytes",
-    "jdb_treelstm_forward_host",
+    "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts",
 ]
 
 
@@ -44,6 +44,11 @@ class COpts(C.Structure):
     _fields_ = [("precision", C.c_int32), ("mode", C.c_int32), ("flags", C.c_int32), ("tuning", C.c_int32),
                 ("barrier_timeout_ns", C.c_uint64), ("ev_begin", C.c_void_p), ("ev_xproj_done", C.c_void_p),
                 ("ev_levels_done", C.c_void_p), ("trace", C.c_void_p), ("trace_cap", C.c_int64)]
+
+
+class CLaunchStats(C.Structure):
+    _fields_ = [("cells_unbatched", C.c_int64), ("cells_batched", C.c_int64), ("ops_unbatched", C.c_int64),
+                ("ops_batched", C.c_int64), ("n_levels", C.c_int32), ("reserved", C.c_int32)]
 
 
 class JdbError(RuntimeError):
@@ -91,6 +96,10 @@ def lib():
     L.jdb_sched_status.argtypes = [C.POINTER(CSched), C.POINTER(i32), C.POINTER(i32), vp]
     L.jdb_debug_report.restype = C.c_int
     L.jdb_debug_report.argtypes = [C.POINTER(CSched), C.POINTER(i32 * 4), vp]
+    L.jdb_launch_counts_workspace_bytes.restype = sz
+    L.jdb_launch_counts_workspace_bytes.argtypes = [i32]
+    L.jdb_launch_counts.restype = C.c_int
+    L.jdb_launch_counts.argtypes = [C.POINTER(CForest), C.POINTER(CSched), C.POINTER(CLaunchStats), vp, sz, vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
     L.jdb_forward_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
     L.jdb_treelstm_forward_host.restype = C.c_int
@@ -253,6 +262,16 @@ def jdb_sched_status(sched: Schedule, stream=None):
     if st != OK:
         raise JdbError(st, "jdb_sched_status")
     return nl.value, nv.value
+
+
+def jdb_launch_counts(forest: Forest, sched: Schedule, ws: Optional[torch.Tensor] = None, stream=None):
+    """(cells_unbatched, cells_batched, ops_unbatched, ops_batched, n_levels): Section 3's launch counts of the forest."""
+    ws = _device_bytes(lib().jdb_launch_counts_workspace_bytes(forest.n_nodes), forest.child_ptr.device) if ws is None else ws
+    cf, cs, out = forest.c(), sched.c(), CLaunchStats()
+    st = lib().jdb_launch_counts(C.byref(cf), C.byref(cs), C.byref(out), _ptr(ws), ws.numel(), _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_launch_counts")
+    return out.cells_unbatched, out.cells_batched, out.ops_unbatched, out.ops_batched, out.n_levels
 
 
 def jdb_debug_report(sched: Schedule, stream=None):

@@ -28,7 +28,7 @@ def test_library_builds_and_exports_every_declared_symbol():
 def test_host_only_queries():
     L = jdb.lib()
     assert L.jdb_status_string(jdb.OK) == b"ok"
-    for code in range(7):
+    for code in range(8):
         assert len(L.jdb_status_string(code)) > 0
     small = L.jdb_schedule_workspace_bytes(1000, 999)
     big = L.jdb_schedule_workspace_bytes(1_600_000, 1_530_000)
@@ -43,8 +43,14 @@ def test_host_only_queries():
     assert hw > fw + 2 * 1000 * 150 * 4
 
 
+def L_places(n):
+    return jdb.lib().jdb_launch_counts_workspace_bytes(n)
+
+
 def test_struct_layouts_match_header():
     # field order and widths as declared in jdb.h (LP64)
     assert ctypes.sizeof(jdb.CForest) == 24
     assert ctypes.sizeof(jdb.CSched) == 48
     assert ctypes.sizeof(jdb.COpts) == 64
+    assert ctypes.sizeof(jdb.CLaunchStats) == 40
+    assert L_places(1) >= 1024 * 8 and L_places(100000) >= 2 * 100000 * 8

@@ -171,9 +171,11 @@ def test_level_ordered_outputs_through_plain_stores_agree_with_tma_stores(monkey
         fixed = np.diff(w.forest.child_ptr) <= 33 if mode == jdb.MODE_PER_LEVEL else np.ones(w.forest.n_nodes, dtype=bool)
         assert np.array_equal(h0[fixed], h1[fixed]) and np.array_equal(c0[fixed], c1[fixed])
         assert np.allclose(h0, h1, rtol=0, atol=2e-6) and np.allclose(c0, c1, rtol=1e-6, atol=2e-6)
-        # the c of a 140-child root is a sum of 140 terms of size up to 1: its error is taken relative to its size
+        # the c of a 140-child root is a sum of 140 terms f c_k, each carrying the logistic approximation's error (up to
+        # 2.6e-4 per term, measured by the test above): its bound grows with the number of children
         ho, co = oracle(w, matched(w, mode))
-        assert np.all(np.abs(h1 - ho) <= TOL_BF16_MATCHED) and np.all(np.abs(c1 - co) <= TOL_BF16_MATCHED + 1e-3 * np.abs(co))
+        fan = np.diff(w.forest.child_ptr).astype(np.float64)[:, None]
+        assert np.all(np.abs(h1 - ho) <= TOL_BF16_MATCHED) and np.all(np.abs(c1 - co) <= TOL_BF16_MATCHED + 2.6e-4 * fan)
 
 
 def sampled_check(index, extra_random, seed, matched_trees=None):
@@ -444,3 +446,57 @@ def test_bf16_degenerate_forests(mode):
         h, c, s = run_forward(w, mode, pad_ld=True)
         assert s.n_levels == (1 if len(parents[0]) == 1 else 131)
         check(w, h, c, TOL_BF16_MATCHED, quantize=matched(w, mode))
+
+
+_DEBUG_CASES = [("fp32", jdb.MODE_PER_LEVEL, 70), ("fp32", jdb.MODE_PERSISTENT, 70), ("fp32", jdb.MODE_PERSISTENT, 200),
+                ("bf16", jdb.MODE_AUTO, 150), ("bf16", jdb.MODE_PER_LEVEL, 150), ("bf16", jdb.MODE_AUTO, 200),
+                ("bf16", jdb.MODE_PERSISTENT, 200)]
+
+
+@pytest.mark.parametrize("precision,mode,H", _DEBUG_CASES)
+def test_debug_checks_pass_on_every_path_and_change_nothing(precision, mode, H):
+    """JDB_FLAG_DEBUG_CHECKS makes every kernel hold the indices it follows against the sizes of the arrays they
+    index.  On a consistent forest and schedule nothing is reported, on every level-loop variant, and the results are
+    the ones of the unchecked run."""
+    parents = [[-1, 0, 0, 1, 1, 1, 2, 5, 5, 5, 5], [-1] + [0] * 40, [-1, 0, 1, 2, 3], [-1], [-1] + list(range(20))] * 30
+    w = wl.make_custom(parents, D=40, H=H, seed=600 + H, precision=precision, bias="random")
+    rng = np.random.default_rng(3)
+    g, new_id = wl.relabel(w.forest, rng)
+    tok = np.empty_like(w.token)
+    tok[new_id] = w.token
+    w.forest, w.token = g, tok
+    h0, c0, _ = run_forward(w, mode, pad_ld=True)
+    h1, c1, s = run_forward(w, mode, pad_ld=True, flags=jdb.FLAG_DEBUG_CHECKS)
+    assert jdb.jdb_debug_report(s)[0] == 0
+    assert np.allclose(h0, h1, rtol=0, atol=2e-6) and np.allclose(c0, c1, rtol=1e-6, atol=2e-6)
+    check(w, h1, c1, TOL_FP32 if precision == "fp32" else TOL_BF16)
+
+
+@pytest.mark.parametrize("precision,mode,H", _DEBUG_CASES)
+def test_debug_checks_report_a_schedule_that_does_not_fit_the_forest(precision, mode, H):
+    """A schedule made for a forest of N nodes, handed in with a forest header that claims N - 7: the schedule's level
+    offsets and node ids then point past what the header allows.  With the checks on, the call reports
+    JDB_ERR_CHECK and names the offender instead of following it.  (Every buffer here is allocated for the full N, so
+    nothing could leave its allocation even unchecked.)"""
+    parents = [[-1, 0, 0, 1, 1, 1, 2, 5, 5, 5, 5], [-1] + [0] * 40, [-1, 0, 1, 2, 3]] * 30
+    w = wl.make_custom(parents, D=40, H=H, seed=700 + H, precision=precision, bias="random")
+    forest, x, packed, prec = device_inputs(w, pad_ld=True)
+    sched = jdb.jdb_schedule(forest)
+    n = forest.n_nodes
+    ws = torch.empty(2 * jdb.forward_workspace(forest, sched, w.D, w.H, prec).numel() + (1 << 20), dtype=torch.uint8, device="cuda")
+    h = torch.zeros((n, w.H + 2), device="cuda")
+    c = torch.zeros_like(h)
+    short = jdb.Forest(forest.child_ptr, forest.child_idx, n - 7, forest.n_edges)
+    with pytest.raises(jdb.JdbError) as ei:
+        jdb.jdb_treelstm_forward(short, sched, x, packed, w.D, w.H, prec, mode=mode, h=h, c=c, ws=ws,
+                                 flags=jdb.FLAG_DEBUG_CHECKS)
+    assert ei.value.status == jdb.ERR_CHECK
+    what, value, bound, where = jdb.jdb_debug_report(sched)
+    assert what != 0 and not (0 <= value < bound)
+    torch.cuda.synchronize()
+    # the same buffers with the true header: clean
+    hh, cc = jdb.jdb_treelstm_forward(forest, sched, x, packed, w.D, w.H, prec, mode=mode, h=h, c=c, ws=ws,
+                                      flags=jdb.FLAG_DEBUG_CHECKS)
+    torch.cuda.synchronize()
+    assert jdb.jdb_debug_report(sched)[0] == 0
+    check(w, hh[:, :w.H].cpu().numpy(), cc[:, :w.H].cpu().numpy(), TOL_FP32 if precision == "fp32" else TOL_BF16)

@@ -163,3 +163,21 @@ def test_argument_errors():
     cfb, csb = big.c(), sb.c()
     ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
     assert L.jdb_schedule(C.byref(cfb), C.byref(csb), C.c_void_p(ws.data_ptr()), 1024, None) == jdb.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("index", [1, 2, 3, 4, 5])
+def test_launch_counts_match_the_checker(index):
+    """Section 3's launch counts at cell and at operator granularity: the GPU count of distinct (depth, number of
+    children) pairs against the one-node-at-a-time checker, on the five workloads and on the hand-counted forest."""
+    from oracle import granularity as og
+    f = wl.make_workload(index).forest
+    forest, s = gpu_schedule(f.child_ptr, f.child_idx)
+    got = jdb.jdb_launch_counts(forest, s)
+    depth = s.depth[:f.n_nodes].cpu().numpy()            # bit-exact against the checker's depths elsewhere in this file
+    assert got == og.launch_counts(f.child_ptr, depth)
+    if index == 1:
+        g = read_golden("forest10.txt")
+        forest, s = gpu_schedule(g["child_ptr"], g["child_idx"])
+        assert list(jdb.jdb_launch_counts(forest, s)) == g["launch_counts"]
+        empty, se = gpu_schedule([0], [])
+        assert jdb.jdb_launch_counts(empty, se) == (0, 0, 0, 0, 0)
