@@ -45,11 +45,16 @@ constexpr int GEMM1_THREADS = 224;  // warp 0: TMA producer, warps 1 and 6: MMA 
 // step), and a scheduler with a single warp issues well below one instruction per cycle: it runs EIGHT epilogue
 // warps, two per TMEM lane quarter and per scheduler, which take the steps of a tile alternately.
 constexpr int GEMMF_THREADS = 320;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
-__host__ __device__ constexpr int gemm_threads(int epi) { return epi == 2 ? GEMMF_THREADS : GEMM1_THREADS; }
+__host__ __device__ constexpr int gemm_threads(int epi) { return (epi == 2 || epi == 3) ? GEMMF_THREADS : GEMM1_THREADS; }
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;
 constexpr int TMEM_COLS = 512;  // two accumulator buffers of up to 256 columns
 
-enum { EPI_XPROJ = 0, EPI_LEVEL = 1, EPI_F = 2 };
+enum { EPI_XPROJ = 0, EPI_LEVEL = 1, EPI_F = 2, EPI_XPROJ8 = 3 };
+// EPI_XPROJ8 is the input projection with eight epilogue warps (used where the bf16 copy of h is kept in child order,
+// i.e. ahead of per-level launches): its epilogue, like the forget-gate one, is bound by how many instructions one
+// warp per scheduler can issue, so two warps per TMEM lane quarter share a tile's steps.
+__host__ __device__ constexpr bool is_xproj(int epi) { return epi == EPI_XPROJ || epi == EPI_XPROJ8; }
+__host__ __device__ constexpr int epi_warps(int epi) { return (epi == EPI_F || epi == EPI_XPROJ8) ? 8 : 4; }
 
 struct TcArgs {
     const int32_t* child_ptr;
@@ -92,7 +97,7 @@ __device__ __forceinline__ Tile tile_of(int t, int n_tiles, int tm, int lo, int 
     Tile r;
     const int m_tile = t / n_tiles;
     r.n_tile = t - m_tile * n_tiles;
-    if (EPI == EPI_XPROJ) {
+    if (is_xproj(EPI)) {
         const bool leaf = m_tile < mt_leaf;
         r.row0 = leaf ? m_tile * tm : n_leaves + (m_tile - mt_leaf) * tm;
         r.row_end = leaf ? n_leaves : hi;
@@ -130,6 +135,9 @@ constexpr int F_RING = 2;   // this step's buffer and the next one's (of the war
 constexpr int F_WARPS = 8;
 constexpr int F_SCRATCH_BYTES = F_WARPS * F_RING * F_STEP_FLOATS * 4;
 constexpr int GEMM_SMEM_F = F_STAGES * STAGE_BYTES + F_SCRATCH_BYTES + 1024;
+constexpr int X8_STAGES = 3;
+constexpr int GEMM_SMEM_X8 = X8_STAGES * STAGE_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;   // eight warps, one step buffer each
+static_assert(GEMM_SMEM_X8 <= 227 * 1024 - 256, "GEMM shared memory");
 static_assert(GEMM_SMEM_STORE <= 227 * 1024 - 256, "GEMM shared memory");
 static_assert(GEMM_SMEM_F <= 227 * 1024 - 256, "forget GEMM shared memory");
 static_assert(GEMM_SMEM_LEVEL <= 227 * 1024 - 256, "level GEMM shared memory");
@@ -320,11 +328,11 @@ __device__ __forceinline__ void xproj_internal_step(const TcArgs& a, const Tile&
 // and lane 0 sends them off as two TMA stores; the load/store units see the staging writes only.  Rows past the last
 // internal node are dropped by the tensor map's bounds (or land in unused rows of P when its row count is a bound).
 __device__ __forceinline__ void xproj_internal_tile_tma(const TcArgs& a, const Tile& ti, const CUtensorMap* tmP, uint32_t taddr,
-                                                        int quarter, int lane, int n_leaves, float* sc) {
+                                                        int quarter, int lane, int n_leaves, float* sc, int k_begin, int k_end) {
     const float* bias = a.bias4;
     const int y = ti.row0 + quarter * 32 - n_leaves;
 #pragma unroll 1
-    for (int k = 0; k < 4; ++k) {
+    for (int k = k_begin; k < k_end; ++k) {  // the planes (i, o, u, f) this warp sends off
         if (lane == 0) bulk_wait_read();  // the stores of the plane before have read the buffer
         __syncwarp();
 #pragma unroll
@@ -599,8 +607,11 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         }
         cp_async_wait<0>();
     } else {
-        // input projection: stores only; every step goes through one step buffer per warp to leave in coalesced pieces
-        float* sc = scratch + quarter * EPI_STEP_FLOATS;
+        // input projection: stores only; every step goes through one step buffer per warp to leave in coalesced pieces.
+        // With eight warps the two warps of a lane quarter take the steps (or the planes of P) alternately.
+        constexpr int NSPLIT = epi_warps(EPI) / 4;
+        const int split = (warp - 2) >> 2;
+        float* sc = scratch + (warp - 2) * EPI_STEP_FLOATS;
         for (int t = t0; t < total_tiles && ok; t += t_step) {
             const Tile ti = tile_at(t);
             const bool leaf = ti.bn == 192;
@@ -614,7 +625,7 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
             tc_fence_after();
             const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
             if (leaf) {
-                if (a.p_tma && !a.child_order) {
+                if (NSPLIT == 1 && a.p_tma && !a.child_order) {
                     // the bf16 copy is kept by position: the tile's rows leave as one TMA store (a plain box).
                     // Rows of a partly filled last leaf tile belong to internal nodes, whose rows are written
                     // again, with their values, by the level that evaluates them.
@@ -630,14 +641,14 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
                     }
                 } else {
 #pragma unroll 1
-                    for (int q = 0; q < 4; ++q) xproj_leaf_step<false>(a, ti, taddr, quarter, lane, q, vs, hbr, sc);
+                    for (int q = split; q < 4; q += NSPLIT) xproj_leaf_step<false>(a, ti, taddr, quarter, lane, q, vs, hbr, sc);
                 }
             } else {
                 if (a.p_tma) {
-                    xproj_internal_tile_tma(a, ti, tmP, taddr, quarter, lane, n_leaves, sc);
+                    xproj_internal_tile_tma(a, ti, tmP, taddr, quarter, lane, n_leaves, sc, split * (4 / NSPLIT), (split + 1) * (4 / NSPLIT));
                 } else {
 #pragma unroll 1
-                    for (int q = 0; q < 4; ++q) xproj_internal_step(a, ti, taddr, quarter, lane, q, n_leaves, sc);
+                    for (int q = split; q < 4; q += NSPLIT) xproj_internal_step(a, ti, taddr, quarter, lane, q, n_leaves, sc);
                 }
             }
             release_acc(acc);
@@ -672,7 +683,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
     // the per-level GEMMs trade one pipeline stage (their K is the hidden size: few blocks) for the epilogue's ring
-    constexpr int NST = EPI == EPI_LEVEL ? LEVEL_STAGES : EPI == EPI_F ? F_STAGES : STAGES;
+    constexpr int NST = EPI == EPI_LEVEL ? LEVEL_STAGES : EPI == EPI_F ? F_STAGES : EPI == EPI_XPROJ8 ? X8_STAGES : STAGES;
     constexpr int SB = EPI == EPI_LEVEL ? LEVEL_STAGE_BYTES : STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[NST], bar_empty[NST], bar_tfull[2], bar_tempty[2];
@@ -690,7 +701,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_tfull[b]), a.issuers);
-            mbar_init(smem_u32(&bar_tempty[b]), EPI == EPI_F ? 32 * F_WARPS : 128);
+            mbar_init(smem_u32(&bar_tempty[b]), 32 * epi_warps(EPI));
         }
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -711,14 +722,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int lo = 0, hi = 0, a_row_off = 0;
     const int n_levels = a.meta[META_N_LEVELS];
     const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
-    if (EPI == EPI_XPROJ) {
+    if (is_xproj(EPI)) {
         hi = a.n_nodes;
     } else if (level < n_levels) {
         level_range<EPI>(a, level, n_leaves, lo, hi);
         a_row_off = (EPI == EPI_LEVEL) ? -n_leaves : 0;
     }
-    const int mt_leaf = EPI == EPI_XPROJ ? (n_leaves + BM - 1) / BM : 0;
-    const int m_tiles = EPI == EPI_XPROJ ? mt_leaf + (hi - n_leaves + BM - 1) / BM : (hi - lo + BM - 1) / BM;
+    const int mt_leaf = is_xproj(EPI) ? (n_leaves + BM - 1) / BM : 0;
+    const int m_tiles = is_xproj(EPI) ? mt_leaf + (hi - n_leaves + BM - 1) / BM : (hi - lo + BM - 1) / BM;
     const int n_tiles = n_total / bn;
     const int total_tiles = m_tiles * n_tiles;
 
@@ -737,8 +748,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (ok) {
                         mbar_expect_tx(full, tx);
                         tma_load_2d(smem_base + stage * SB, &tmA, full, kb * BK, ti.row0 + a_row_off);
-                        tma_load_2d(smem_base + stage * SB + A_BYTES, (EPI == EPI_XPROJ && ti.bn == 192) ? &tmB_leaf : &tmB,
-                                    full, kb * BK, EPI == EPI_XPROJ ? ti.n_tile * 256 : ti.n_tile * bn);
+                        tma_load_2d(smem_base + stage * SB + A_BYTES, (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB,
+                                    full, kb * BK, is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -747,7 +758,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
         if (!ok && lane == 0) *abort = 1;
-    } else if (warp == 1 || (EPI != EPI_F && warp == 6 && a.issuers == 2)) {
+    } else if (warp == 1 || (epi_warps(EPI) == 4 && warp == 6 && a.issuers == 2)) {
         // One MMA issuer for the whole tile width, or two taking half of the columns each.  The whole warp walks the pipeline (waits,
         // descriptors), so every operand of tcgen05.mma is warp-uniform; one elected lane issues.
         {
@@ -787,7 +798,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (!ok && lane == 0) *abort = 1;
         }
-    } else if (warp >= 2 && warp <= (EPI == EPI_F ? 1 + F_WARPS : 5)) {
+    } else if (warp >= 2 && warp <= 1 + epi_warps(EPI)) {
         epilogue_warps<EPI, false>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST * SB), tmem_base,
                                    bar_tfull, bar_tempty, abort, warp, lane, blockIdx.x, gridDim.x, total_tiles, n_tiles, lo, hi,
                                    bn, n_leaves, mt_leaf, 0);
@@ -815,6 +826,7 @@ constexpr int STAGE2_BYTES = A_BYTES + B_BYTES_MAX / 2;
 constexpr int GEMM2_SMEM = STAGES2 * STAGE2_BYTES + 4 * EPI_STEP_FLOATS * 4 + 1024;
 constexpr int GEMM2_SMEM_LEVEL = STAGES2_LEVEL * STAGE2_BYTES + EPI_SCRATCH_BYTES + 1024;
 constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH_BYTES + 1024;
+constexpr int GEMM2_SMEM_X8 = STAGES2_LEVEL * STAGE2_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;
 static_assert(GEMM2_SMEM_LEVEL <= 227 * 1024 - 256, "pair level GEMM shared memory");
 
 template <int EPI>
@@ -822,7 +834,7 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
-    constexpr int NST2 = EPI == EPI_XPROJ ? STAGES2 : STAGES2_LEVEL;
+    constexpr int NST2 = EPI == EPI_XPROJ ? STAGES2 : STAGES2_LEVEL;   // the kernels with rings or eight step buffers give up two stages
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[NST2], bar_empty[NST2], bar_tfull[2], bar_tempty[2];
     __shared__ uint32_t s_tmem_base;
@@ -838,7 +850,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     int lo, hi, a_row_off;
     const int n_levels = a.meta[META_N_LEVELS];
     const int n_leaves = n_levels > 0 ? a.level_ptr[1] : 0;
-    if (EPI == EPI_XPROJ) {
+    if (is_xproj(EPI)) {
         lo = 0; hi = a.n_nodes; a_row_off = 0;
     } else {
         if (level >= n_levels) return;  // uniform over the whole grid; nothing allocated, no cluster barrier yet
@@ -846,8 +858,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         a_row_off = (EPI == EPI_LEVEL) ? -n_leaves : 0;
     }
     constexpr int TM2 = 2 * BM;
-    const int mt_leaf = EPI == EPI_XPROJ ? (n_leaves + TM2 - 1) / TM2 : 0;
-    const int m_tiles = EPI == EPI_XPROJ ? mt_leaf + (hi - n_leaves + TM2 - 1) / TM2 : (hi - lo + TM2 - 1) / TM2;
+    const int mt_leaf = is_xproj(EPI) ? (n_leaves + TM2 - 1) / TM2 : 0;
+    const int m_tiles = is_xproj(EPI) ? mt_leaf + (hi - n_leaves + TM2 - 1) / TM2 : (hi - lo + TM2 - 1) / TM2;
     const int n_tiles = n_total / bn;
     const int total_tiles = m_tiles * n_tiles;
 
@@ -859,7 +871,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_tfull[b]), 1);
-            mbar_init(smem_u32(&bar_tempty[b]), EPI == EPI_F ? 64 * F_WARPS : 256);  // the epilogue threads of both CTAs
+            mbar_init(smem_u32(&bar_tempty[b]), 64 * epi_warps(EPI));  // the epilogue threads of both CTAs
         }
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -890,8 +902,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[stage]), tx);
                         tma_load_2d_pair(smem_base + stage * STAGE2_BYTES, &tmA, full_leader, kb * BK, my_row0 + a_row_off);
                         // this CTA's half of the B tile's rows (the MMA reads rows 0.. from CTA 0, the rest from CTA 1)
-                        const int n_base = EPI == EPI_XPROJ ? ti.n_tile * 256 : ti.n_tile * bn;
-                        const CUtensorMap* tb = (EPI == EPI_XPROJ && ti.bn == 192) ? &tmB_leaf : &tmB;
+                        const int n_base = is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn;
+                        const CUtensorMap* tb = (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB;
                         tma_load_2d_pair(smem_base + stage * STAGE2_BYTES + A_BYTES, tb, full_leader, kb * BK,
                                          n_base + (int)rank * half_bn);
                     }
@@ -940,7 +952,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             if (!ok && lane == 0) *abort = 1;
         }
-    } else if (warp >= 2 && warp <= (EPI == EPI_F ? 1 + F_WARPS : 5)) {
+    } else if (warp >= 2 && warp <= 1 + epi_warps(EPI)) {
         epilogue_warps<EPI, true>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST2 * STAGE2_BYTES),
                                   tmem_base, bar_tfull, bar_tempty, abort, warp, lane, pair, n_pairs, total_tiles, n_tiles, lo, hi,
                                   bn, n_leaves, mt_leaf, (int)rank);
@@ -1249,6 +1261,7 @@ bool make_tmap_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t col
 struct Tuning {
     int pair_mask, issuers;
     bool pdl, p_tma;
+    bool issuers2_requested;   // two MMA issuers exist only in the kernels with four epilogue warps
 };
 Tuning resolve_tuning(int32_t t) {
     Tuning r;
@@ -1257,6 +1270,7 @@ Tuning resolve_tuning(int32_t t) {
         r.issuers = (t & JDB_TUNE_TWO_ISSUERS) ? 2 : 1;
         r.pdl = !(t & JDB_TUNE_NO_PDL);
         r.p_tma = !(t & JDB_TUNE_PLAIN_STORES);
+        r.issuers2_requested = r.issuers == 2;
         return r;
     }
     const char* e = getenv("JDB_GEMM_PAIR");
@@ -1267,6 +1281,7 @@ Tuning resolve_tuning(int32_t t) {
     r.pdl = !(e && e[0] == '0');
     e = getenv("JDB_P_TMA");
     r.p_tma = !(e && e[0] == '0');
+    r.issuers2_requested = r.issuers == 2;
     return r;
 }
 
@@ -1413,6 +1428,8 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_XPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_STORE));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_LEVEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_LEVEL));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_F>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_F));
+        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI_XPROJ8>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_X8));
+        JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_XPROJ8>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM_X8));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_XPROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_LEVEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM_LEVEL));
         JDB_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI_F>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM2_SMEM_F));
@@ -1433,11 +1450,12 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         const int n_tiles = n_total / bn;
         // the forget-gate GEMM decides launch by launch: pairs pay off from about 32 tiles per pair on
         const long long tiles2 = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles;
-        const bool pair = epi == EPI_XPROJ ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_f && tiles2 >= 32LL * (n_sm / 2));
+        const bool pair = is_xproj(epi) ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_f && tiles2 >= 32LL * (n_sm / 2));
         const CUtensorMap& tB = (epi == EPI_F && pair) ? tmUfH : tB_full;
         if (!pair) {
             const int grid = gemm_grid(rows_bound, n_tiles);
             if (epi == EPI_XPROJ) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+            else if (epi == EPI_XPROJ8) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ8>, dim3(grid), dim3(GEMMF_THREADS), GEMM_SMEM_X8, st, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
             else if (epi == EPI_LEVEL) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_LEVEL>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_LEVEL, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
             else JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_F>, dim3(grid), dim3(GEMMF_THREADS), GEMM_SMEM_F, st, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
             return JDB_OK;
@@ -1446,7 +1464,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(2 * pairs);
         cfg.blockDim = dim3(gemm_threads(epi));
-        cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : epi == EPI_F ? GEMM2_SMEM_F : GEMM2_SMEM;
+        cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : epi == EPI_F ? GEMM2_SMEM_F : epi == EPI_XPROJ8 ? GEMM2_SMEM_X8 : GEMM2_SMEM;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1458,6 +1476,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         cfg.attrs = attr;
         cfg.numAttrs = tune.pdl ? 2 : 1;
         if (epi == EPI_XPROJ) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_XPROJ>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
+        else if (epi == EPI_XPROJ8) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_XPROJ8>, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
         else if (epi == EPI_LEVEL) JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_LEVEL>, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
         else JDB_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI_F>, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
         return JDB_OK;
@@ -1481,7 +1500,11 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         edge_fill_kernel<<<(int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16), 256, 0, st>>>(a, w.block_sum);
         JDB_CUDA_TRY(cudaGetLastError());
     }
-    if ((ls = launch(EPI_XPROJ, tmX, tmW, tmWl, (long long)N + 2 * BM, 0, 256, 4 * Hp, kd)) != JDB_OK) return ls;
+    // eight epilogue warps where the bf16 copy of h goes out row by row anyway (child order) and the forest is large
+    // enough for the epilogue to matter; the small forests of the cooperative loop keep the four-warp kernel, whose
+    // leaf tiles leave as one TMA box per warp
+    const int xepi = (!use_small && !tune.issuers2_requested) ? EPI_XPROJ8 : EPI_XPROJ;
+    if ((ls = launch(xepi, tmX, tmW, tmWl, (long long)N + 2 * BM, 0, 256, 4 * Hp, kd)) != JDB_OK) return ls;
     if (fa.ev_xproj_done) JDB_CUDA_TRY(cudaEventRecord(fa.ev_xproj_done, st));
     if (!use_small) {
         const int cs_blocks = (int)((ni + 7) / 8 < (size_t)n_sm * 8 ? (ni + 7) / 8 : (size_t)n_sm * 8);
