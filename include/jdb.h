@@ -56,7 +56,7 @@ enum {
 };
 
 /* jdb_opts.tuning: 0 takes the library's defaults (the measured best, which the environment variables JDB_GEMM_PAIR,
- * JDB_GEMM_ISSUERS, JDB_PDL and JDB_P_TMA may change, read at every call).  With JDB_TUNE_SET the other bits
+ * JDB_GEMM_ISSUERS, JDB_PDL, JDB_P_TMA and JDB_GATHER_X may change, read at every call).  With JDB_TUNE_SET the other bits
  * replace those defaults for this call; every combination computes the same values. */
 enum {
     JDB_TUNE_SET = 1,
@@ -65,7 +65,9 @@ enum {
     JDB_TUNE_PAIR_FORGET = 8,   /* per-level forget-gate GEMM as CTA pairs (launches with at least 32 tiles per pair)*/
     JDB_TUNE_TWO_ISSUERS = 16,  /* two MMA-issuing warps per lone CTA, half of the tile's columns each               */
     JDB_TUNE_NO_PDL = 32,       /* ordinary launches instead of programmatic dependent launches                      */
-    JDB_TUNE_PLAIN_STORES = 64  /* level-ordered outputs through the load/store units instead of TMA stores           */
+    JDB_TUNE_PLAIN_STORES = 64, /* level-ordered outputs through the load/store units instead of TMA stores           */
+    JDB_TUNE_GATHER_X = 128     /* bf16 x with 16-byte aligned rows is read in place by the input projection (TMA row
+                                   gathers keyed by perm) instead of being laid out in level order first; slower      */
 };
 
 #define JDB_META_INTS 16 /* size of jdb_sched.meta in int32 */

@@ -84,6 +84,7 @@ struct TcArgs {
     int32_t* slot_par;    // [n_edges]         row (position - n_leaves) of the parent that owns the slot
     int32_t* slot_child;  // [n_edges]         node id of the child at the slot
     int32_t debug;        // check every index against its array before following it
+    int32_t x_gather;     // the input projection reads its rows straight from the caller's x, picked by perm (TMA row gather)
 };
 
 // Where a tile sits.  The input projection walks the rows in level order and never mixes
@@ -734,26 +735,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int total_tiles = m_tiles * n_tiles;
 
     if (warp == 0) {
-        // producer warp: lane 0 waits for the stage and issues both tile loads
+        // producer warp: lane 0 waits for the stage and issues the tile loads.  With x_gather the rows of the input
+        // projection's A tile are rows of the caller's x picked by perm: every lane holds four of the tile's node ids
+        // and issues one four-row gather per K block (rows past the tile's end repeat its last row; nobody reads them).
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
+        const bool gather = is_xproj(EPI) && a.x_gather;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const Tile ti = tile_of<EPI>(t, n_tiles, BM, lo, hi, bn, n_leaves, mt_leaf);
             const uint32_t tx = A_BYTES + (uint32_t)ti.bn * BK * 2;
+            int rows[4] = {0, 0, 0, 0};
+            if (gather) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int p = min(ti.row0 + 4 * lane + i, ti.row_end - 1);
+                    int v = a.perm[p];
+                    if (a.debug && !dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, p)) v = 0;
+                    rows[i] = v;
+                }
+            }
             for (int kb = 0; kb < kblocks; ++kb) {
                 const uint32_t full = smem_u32(&bar_full[stage]);
                 if (lane == 0) {
                     ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort);
                     if (ok) {
                         mbar_expect_tx(full, tx);
-                        tma_load_2d(smem_base + stage * SB, &tmA, full, kb * BK, ti.row0 + a_row_off);
+                        if (!gather) tma_load_2d(smem_base + stage * SB, &tmA, full, kb * BK, ti.row0 + a_row_off);
                         tma_load_2d(smem_base + stage * SB + A_BYTES, (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB,
                                     full, kb * BK, is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                if (gather) tma_gather4_2d(smem_base + stage * SB + lane * 512, &tmA, full, kb * BK, rows[0], rows[1], rows[2], rows[3]);
                 if (++stage == NST) { stage = 0; phase ^= 1u; }
             }
         }
@@ -889,18 +904,29 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
+        const bool gather = is_xproj(EPI) && a.x_gather;
         for (int t = pair; t < total_tiles && ok; t += n_pairs) {
             const Tile ti = tile_of<EPI>(t, n_tiles, TM2, lo, hi, bn, n_leaves, mt_leaf);
             const int half_bn = ti.bn >> 1;
             const uint32_t tx = 2u * (A_BYTES + (uint32_t)half_bn * BK * 2);
             const int my_row0 = ti.row0 + (int)rank * BM;
+            int rows[4] = {0, 0, 0, 0};   // x_gather: node ids of the four rows this lane fetches (see the lone-CTA kernel)
+            if (gather) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int p = min(my_row0 + 4 * lane + i, ti.row_end - 1);
+                    int v = a.perm[p];
+                    if (a.debug && !dbg_ok(a.meta, CHECK_PERM, v, a.n_nodes, p)) v = 0;
+                    rows[i] = v;
+                }
+            }
             for (int kb = 0; kb < kblocks; ++kb) {
                 const uint32_t full_leader = mapa_u32(smem_u32(&bar_full[stage]), 0);
                 if (lane == 0) {
                     ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort);
                     if (ok) {
                         if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[stage]), tx);
-                        tma_load_2d_pair(smem_base + stage * STAGE2_BYTES, &tmA, full_leader, kb * BK, my_row0 + a_row_off);
+                        if (!gather) tma_load_2d_pair(smem_base + stage * STAGE2_BYTES, &tmA, full_leader, kb * BK, my_row0 + a_row_off);
                         // this CTA's half of the B tile's rows (the MMA reads rows 0.. from CTA 0, the rest from CTA 1)
                         const int n_base = is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn;
                         const CUtensorMap* tb = (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB;
@@ -910,6 +936,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                if (gather) tma_gather4_2d_pair(smem_base + stage * STAGE2_BYTES + lane * 512, &tmA, full_leader, kb * BK, rows[0], rows[1], rows[2], rows[3]);
                 if (++stage == NST2) { stage = 0; phase ^= 1u; }
             }
         }
@@ -1182,6 +1209,18 @@ __global__ void __launch_bounds__(256) level_order_x_kernel(const void* __restri
     }
 }
 
+// Position of every node in level order (the inverse of perm), for forwards that do not copy x.
+__global__ void __launch_bounds__(256) inverse_perm_kernel(const int32_t* __restrict__ perm, int N, int32_t* __restrict__ inv,
+                                                           int32_t* meta, int debug) {
+    griddep_wait();
+    griddep_launch();
+    for (int pos = blockIdx.x * blockDim.x + threadIdx.x; pos < N; pos += gridDim.x * blockDim.x) {
+        const int v = perm[pos];
+        if (debug && !dbg_ok(meta, CHECK_PERM, v, N, pos)) continue;
+        inv[v] = pos;
+    }
+}
+
 // ---- weight packing for the tensor-core path -----------------------------------------------------------
 // Rows of B are output features; each 64-wide hidden slice keeps its gates next to each other so that one
 // accumulator tile holds every gate of the same hidden indices: row n of a G-gate matrix maps to
@@ -1262,6 +1301,7 @@ struct Tuning {
     int pair_mask, issuers;
     bool pdl, p_tma;
     bool issuers2_requested;   // two MMA issuers exist only in the kernels with four epilogue warps
+    bool gather_x;             // read x in place through TMA row gathers instead of laying it out in level order first
 };
 Tuning resolve_tuning(int32_t t) {
     Tuning r;
@@ -1271,6 +1311,7 @@ Tuning resolve_tuning(int32_t t) {
         r.pdl = !(t & JDB_TUNE_NO_PDL);
         r.p_tma = !(t & JDB_TUNE_PLAIN_STORES);
         r.issuers2_requested = r.issuers == 2;
+        r.gather_x = (t & JDB_TUNE_GATHER_X) != 0;
         return r;
     }
     const char* e = getenv("JDB_GEMM_PAIR");
@@ -1282,6 +1323,8 @@ Tuning resolve_tuning(int32_t t) {
     e = getenv("JDB_P_TMA");
     r.p_tma = !(e && e[0] == '0');
     r.issuers2_requested = r.issuers == 2;
+    e = getenv("JDB_GATHER_X");
+    r.gather_x = e && e[0] == '1';
     return r;
 }
 
@@ -1401,8 +1444,13 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     a.issuers = tune.issuers;
     a.p_tma = tune.p_tma ? 1 : 0;
 
-    // x goes into level order (and bf16) once; the copy reads 16-byte pieces when x is bf16 with aligned rows
+    // x goes into level order (and bf16) once, in a pass of its own; the copy reads 16-byte pieces when x is bf16 with
+    // aligned rows.  Such an x can instead be read in place, its rows picked by perm through TMA row gathers
+    // (JDB_TUNE_GATHER_X): correct, but every K block of every tile then costs 32 four-row gathers instead of one
+    // box load, and the copy engine does not keep up (workload 5 projection 28.8 ms instead of 11.8, workload 3
+    // 0.79 instead of 0.44), so it is off unless asked for.
     const int x_vec = fa.x_is_bf16 && (fa.ldx % 8 == 0) && (((uintptr_t)fa.x & 15) == 0);
+    a.x_gather = (x_vec && tune.gather_x) ? 1 : 0;
     // CTA pairs pay off once there are enough 256-row tiles to keep every pair busy; below that the lone-CTA
     // kernel has the shorter tail.  In pair mode every CTA loads half of a B tile, so the B maps have half-height boxes.
     const bool big = !use_small && (long long)N >= 2LL * BM * n_sm;
@@ -1411,7 +1459,8 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmUf, tmUfH, tmP, tmHBs;
     const int bnf = g_bn(Hp);
     // W is read through a full box and a leaf box (i, o, u blocks only)
-    bool ok = make_tmap(&tmX, w.xb, n, (uint64_t)D, (uint64_t)Dp, BM) &&
+    bool ok = (a.x_gather ? make_tmap(&tmX, fa.x, n, (uint64_t)D, (uint64_t)fa.ldx, 1)    // one-row boxes for the gathers
+                          : make_tmap(&tmX, w.xb, n, (uint64_t)D, (uint64_t)Dp, BM)) &&
               make_tmap(&tmW, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 256 / bdiv) &&
               make_tmap(&tmWl, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 192 / bdiv);
     if (ok && !use_small)   // the per-level launches read their operands through five more maps
@@ -1484,7 +1533,11 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
 
     jdb_status ls = JDB_OK;
     if (fa.ev_begin) JDB_CUDA_TRY(cudaEventRecord(fa.ev_begin, st));
-    {
+    if (a.x_gather) {
+        const long long want = ((long long)N + 255) / 256;
+        const int blocks = (int)(want < (long long)n_sm * 8 ? want : (long long)n_sm * 8);
+        JDB_CUDA_TRY(launch_behind(tune.pdl, inverse_perm_kernel, dim3(blocks), dim3(256), 0, st, fa.perm, N, w.inv, fa.meta, (int)fa.debug));
+    } else {
         const long long want = ((long long)N + 7) / 8;
         const int blocks = (int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16);
         JDB_CUDA_TRY(launch_behind(tune.pdl, level_order_x_kernel, dim3(blocks), dim3(256), 0, st, fa.x, (int)fa.x_is_bf16, fa.ldx, fa.perm, N, D, Dp,

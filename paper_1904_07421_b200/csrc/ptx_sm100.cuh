@@ -98,6 +98,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// Four rows of a 2-D tensor, picked by index, into four consecutive 128-byte rows of shared memory (the tensor map's
+// box is one row high).  The map covers this GPU's own memory; no multicast.
+__device__ __forceinline__ void tma_gather4_2d(uint32_t dst, const void* tmap, uint32_t bar, int x, int y0, int y1, int y2, int y3) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
+        : "memory");
+}
 // Tiled TMA store shared memory -> global memory of one box at coordinates (x, y), tracked by the issuing thread's
 // bulk group.  x times the element size must be a multiple of 16 bytes; rows and columns past the tensor are dropped.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int x, int y) {
@@ -227,6 +235,12 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap,
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tmap), "r"(bar_cluster), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_gather4_2d_pair(uint32_t dst, const void* tmap, uint32_t bar_cluster, int x, int y0, int y1, int y2, int y3) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar_cluster), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
         : "memory");
 }
 // one MMA over the pair: A rows and accumulator rows split 128/128 between the CTAs, each CTA holds half of B's rows

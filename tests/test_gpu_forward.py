@@ -242,7 +242,9 @@ _TUNINGS = [jdb.TUNE_SET,                                                       
             jdb.TUNE_SET | jdb.TUNE_PAIR_XPROJ | jdb.TUNE_PAIR_LEVEL | jdb.TUNE_PAIR_FORGET,   # CTA pairs wherever allowed
             jdb.TUNE_SET | jdb.TUNE_PAIR_FORGET | jdb.TUNE_TWO_ISSUERS,
             jdb.TUNE_SET | jdb.TUNE_PAIR_FORGET | jdb.TUNE_NO_PDL,
-            jdb.TUNE_SET | jdb.TUNE_PAIR_XPROJ | jdb.TUNE_PLAIN_STORES]
+            jdb.TUNE_SET | jdb.TUNE_PAIR_XPROJ | jdb.TUNE_PLAIN_STORES,
+            jdb.TUNE_SET | jdb.TUNE_PAIR_FORGET | jdb.TUNE_GATHER_X,
+            jdb.TUNE_SET | jdb.TUNE_PAIR_XPROJ | jdb.TUNE_GATHER_X | jdb.TUNE_TWO_ISSUERS]
 
 
 
