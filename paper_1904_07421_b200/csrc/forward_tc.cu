@@ -12,9 +12,10 @@
 //              node sits at the slot of the edge that leads to it, edges numbered by (position of the parent in
 //              level order, index in the parent's child list).  The children of a level's nodes are therefore one
 //              contiguous range of rows, sorted by parent: the product U_f h_k over them is a plain GEMM with TMA
-//              operands, and its epilogue turns every row into f_jk c_k = sig(W_f x_j + b_f + U_f h_k) c_k and adds
-//              the rows of one parent up (a segmented sum over the accumulator rows), so that only
-//              S_j = sum_k f_jk c_k, one row per PARENT, leaves the kernel.
+//              operands.  It is computed TRANSPOSED, hidden units along the accumulator rows and edges along its
+//              columns, so that a thread owns one hidden unit and meets the edges of a parent one after the other:
+//              the epilogue turns every value into f_jk c_k = sig(W_f x_j + b_f + U_f h_k) c_k and adds the values of
+//              one parent up in a register, and only S_j = sum_k f_jk c_k, one row per PARENT, leaves the kernel.
 //   EPI_LEVEL  one level: (i, o, u) pre-activations = P + U_iou h~ with h~ the child sums; the epilogue adds
 //              S_j and finishes c_j = i u + S_j, h_j = o tanh(c_j), and files the bf16 copy of h_j at its slot.
 //
@@ -132,9 +133,12 @@ constexpr int GEMM_SMEM_STORE = GEMM_SMEM + 4 * EPI_STEP_FLOATS * 4;   // input 
 // arrays (the parent's forget pre-activation and the child's c)
 constexpr int F_STEP_FLOATS = 2 * 32 * 16;
 constexpr int F_STAGES = 3;
-constexpr int F_RING = 2;   // this step's buffer and the next one's (of the warp's own steps, which are every other step)
 constexpr int F_WARPS = 8;
-constexpr int F_SCRATCH_BYTES = F_WARPS * F_RING * F_STEP_FLOATS * 4;
+// step buffers per warp: the copies of a step start F_RING - 1 steps ahead.  A CTA of a pair holds half of B per
+// stage, which leaves room for one more buffer per warp than a lone CTA has.
+__host__ __device__ constexpr int f_ring(bool pair) { return pair ? 3 : 2; }
+constexpr int F_SCRATCH_BYTES = F_WARPS * f_ring(false) * F_STEP_FLOATS * 4;
+constexpr int F_SCRATCH2_BYTES = F_WARPS * f_ring(true) * F_STEP_FLOATS * 4;
 constexpr int GEMM_SMEM_F = F_STAGES * STAGE_BYTES + F_SCRATCH_BYTES + 1024;
 constexpr int X8_STAGES = 3;
 constexpr int GEMM_SMEM_X8 = X8_STAGES * STAGE_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;   // eight warps, one step buffer each
@@ -369,27 +373,33 @@ __device__ __forceinline__ void xproj_internal_tile_tma(const TcArgs& a, const T
 }
 
 // ---- epilogue of a forget-gate tile ---------------------------------------------------------------------------
-// Rows of the tile are edge slots, sorted by parent.  Per 16-column step a warp needs, for each of its 32 rows, the
-// parent's forget pre-activation P_f[parent] and the child's c_k: both arrive through the same kind of ring as the
-// level tile's P and S slices (four lanes per row, 16-byte asynchronous copies, two steps ahead).
-// pr, kd: parent row and child node id of tile rows (lane >> 2) + 8 i of this warp (-1: no such row).
-__device__ __forceinline__ void forget_fetch(const TcArgs& a, const Tile& ti, int lane, int q, const int (&pr)[4],
-                                             const int (&kd)[4], uint32_t buf, float* bufp) {
-    const int col = ti.n_tile * ti.bn + q * 16 + (lane & 3) * 4;
+// The accumulator holds (hidden unit, edge): TMEM lane = hidden unit, column = edge slot, 256 edges per tile, sorted by
+// parent.  A warp owns 32 hidden units (its lane quarter) and a segment of 128 consecutive edges, walked in eight
+// steps of 16 edges.  Per step it needs, for each edge, 32 floats of the parent's forget pre-activation P_f and of
+// the child's c: [16 edges][32 floats] arrays in shared memory, filled by 16-byte asynchronous copies one step ahead
+// (eight lanes per edge row) and read one float per lane, free of bank conflicts.
+constexpr int F_EDGES = 256;      // edges per tile (the MMA's N)
+constexpr int F_SEG = 128;        // edges per epilogue warp
+// pr, kd: parent row and child node id of this lane's edges lane + 32 i of the segment, chosen for the step by the caller
+__device__ __forceinline__ void forget_fetch(const TcArgs& a, int j_base, int lane, int st, int pr_sel, int kd_sel, uint32_t buf,
+                                             float* bufp) {
+    const int chunk = lane & 7, col = j_base + chunk * 4;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = (lane >> 2) + 8 * i;
-        const int o = sw_off(row, lane & 3);
+    for (int k = 0; k < 4; ++k) {
+        const int er = (lane >> 3) + 4 * k;                       // edge row of the step
+        const int src_lane = (st & 1) * 16 + er;                  // the lane that holds this edge's parent and child
+        const int par = __shfl_sync(0xffffffffu, pr_sel, src_lane), kid = __shfl_sync(0xffffffffu, kd_sel, src_lane);
+        const int o = er * 32 + chunk * 4;
         const uint32_t d = buf + (uint32_t)o * 4;
-        const bool have = pr[i] >= 0;
-        cp_async16_ca_zfill(d, have ? a.P + ((size_t)pr[i] * 4 + 3) * a.Hp + col : a.P, have ? 16u : 0u);
+        const bool have = par >= 0 && col < a.Hp;
+        cp_async16_ca_zfill(d, have ? a.P + ((size_t)par * 4 + 3) * a.Hp + col : a.P, have ? 16u : 0u);
         const int left = have ? a.H - col : 0;   // columns of the child's c row from `col` on
         if (left >= 4 && a.vec_ok) {
-            cp_async16_zfill(d + 2048, a.c + (int64_t)kd[i] * a.ldh + col, 16u);
+            cp_async16_zfill(d + 2048, a.c + (int64_t)kid * a.ldh + col, 16u);
         } else if (left <= 0) {
             cp_async16_zfill(d + 2048, a.P, 0u);
         } else {  // ragged end of the row, or rows that are not 16-byte aligned
-            const float* src = a.c + (int64_t)kd[i] * a.ldh + col;
+            const float* src = a.c + (int64_t)kid * a.ldh + col;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             v.x = __ldcg(src);
             if (left > 1) v.y = __ldcg(src + 1);
@@ -400,58 +410,80 @@ __device__ __forceinline__ void forget_fetch(const TcArgs& a, const Tile& ti, in
     }
 }
 
-// How this warp's 32 rows fall into runs of equal parent: distance of a lane from the first lane of its run, whether it
-// is the last lane of its run, and how many doubling steps the longest run needs.
-struct Runs {
-    int dist, steps;
-    bool last;
+// What a warp knows about its segment of a tile.
+struct Segment {
+    int pr[4], kd[4];        // parent row / child id of edges lane + 32 i (-1: no such edge)
+    unsigned heads[4];       // bit e of word i: edge 32 i + e starts a new parent
+    bool cont_before;        // the first parent's children start before this segment
+    bool cont_after;         // the last parent's children go on behind this segment
 };
-__device__ __forceinline__ Runs runs_of(int par, int lane) {
-    const int prev = __shfl_up_sync(0xffffffffu, par, 1), next = __shfl_down_sync(0xffffffffu, par, 1);
-    const unsigned heads = __ballot_sync(0xffffffffu, lane == 0 || prev != par);
-    Runs r;
-    r.dist = lane - (31 - __clz(heads & (0xffffffffu >> (31 - lane))));
-    r.last = lane == 31 || next != par;
-    const int longest = __reduce_max_sync(0xffffffffu, r.dist);
-    r.steps = longest == 0 ? 0 : 32 - __clz(longest);
-    return r;
-}
+__device__ __forceinline__ int sel4(const int (&v)[4], int i) { return i == 0 ? v[0] : i == 1 ? v[1] : i == 2 ? v[2] : v[3]; }
+__device__ __forceinline__ unsigned sel4u(const unsigned (&v)[4], int i) { return i == 0 ? v[0] : i == 1 ? v[1] : i == 2 ? v[2] : v[3]; }
 
-// One 16-column step: f c_k for this lane's row, added up over the lanes of the same parent (an inclusive scan in
-// doubling steps that never crosses a run boundary), and the run totals added into S.  A parent whose children
-// straddle warps or tiles receives one contribution from each: S starts at zero and takes them by atomic adds.
-__device__ __forceinline__ void forget_step(const TcArgs& a, const Tile& ti, uint32_t taddr, int lane, int q, int par,
-                                            const Runs& runs, const float* sc) {
-    float g[16];
-    tmem_ld16(taddr + q * 16, g);
-    tmem_ld_wait();
-    float fc[16];
+__device__ __forceinline__ Segment segment_of(const TcArgs& a, int slot0, int row_end, int lane) {
+    Segment sg;
 #pragma unroll
-    for (int c4 = 0; c4 < 4; ++c4) {
-        const int o = sw_off(lane, c4);
-        const float4 pf = *reinterpret_cast<const float4*>(sc + o), ck = *reinterpret_cast<const float4*>(sc + 512 + o);
-        fc[4 * c4 + 0] = sigmoid_fast(pf.x + g[4 * c4 + 0]) * ck.x;
-        fc[4 * c4 + 1] = sigmoid_fast(pf.y + g[4 * c4 + 1]) * ck.y;
-        fc[4 * c4 + 2] = sigmoid_fast(pf.z + g[4 * c4 + 2]) * ck.z;
-        fc[4 * c4 + 3] = sigmoid_fast(pf.w + g[4 * c4 + 3]) * ck.w;
-    }
-    __syncwarp();  // every lane has read its inputs: the buffer may be refilled
-#pragma unroll 1
-    for (int k = 0; k < runs.steps; ++k) {
-        const int off = 1 << k;
-        const bool take = runs.dist >= off;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float up = __shfl_up_sync(0xffffffffu, fc[i], off);
-            if (take) fc[i] += up;
+    for (int i = 0; i < 4; ++i) {
+        const int sl = slot0 + 32 * i + lane;
+        sg.pr[i] = sg.kd[i] = -1;
+        if (sl < row_end) {
+            sg.pr[i] = a.slot_par[sl];
+            sg.kd[i] = a.slot_child[sl];
+            if (a.debug && (!dbg_ok(a.meta, CHECK_PARENT_ROW, sg.pr[i], a.n_int_bound, sl) ||
+                            !dbg_ok(a.meta, CHECK_CHILD, sg.kd[i], a.n_nodes, sl)))
+                sg.pr[i] = sg.kd[i] = -1;
         }
     }
-    if (runs.last && par >= 0) {
-        float* dst = a.S + (size_t)par * a.Hp + ti.n_tile * ti.bn + q * 16;
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * c4), "f"(fc[4 * c4]), "f"(fc[4 * c4 + 1]),
-                         "f"(fc[4 * c4 + 2]), "f"(fc[4 * c4 + 3]) : "memory");
+    for (int i = 0; i < 4; ++i) {
+        int prev = __shfl_up_sync(0xffffffffu, sg.pr[i], 1);
+        const int carry = __shfl_sync(0xffffffffu, sg.pr[i > 0 ? i - 1 : 0], 31);
+        if (lane == 0) prev = carry;
+        sg.heads[i] = __ballot_sync(0xffffffffu, (i == 0 && lane == 0) || sg.pr[i] != prev);
+    }
+    const int n_valid = min(max(row_end - slot0, 0), F_SEG);
+    const int p_first = __shfl_sync(0xffffffffu, sg.pr[0], 0);
+    sg.cont_before = p_first >= 0 && a.eoff[p_first] != slot0;
+    sg.cont_after = false;
+    if (n_valid == F_SEG) {
+        const int p_last = __shfl_sync(0xffffffffu, sg.pr[3], 31);
+        sg.cont_after = p_last >= 0 && a.eoff[p_last + 1] != slot0 + F_SEG;
+    }
+    return sg;
+}
+
+// The running sum of one parent's f c_k in this thread's hidden unit, and where it goes when the parent's edges end:
+// a plain store if all of the parent's edges lie in this segment, else an atomic addition (S starts at zero; a parent
+// whose children straddle segments receives one contribution from each).
+struct RunSum {
+    float sum;
+    int par, runs_done;
+};
+__device__ __forceinline__ void run_flush(const TcArgs& a, const RunSum& r, int j, bool j_ok, bool partial) {
+    if (r.par < 0 || !j_ok) return;
+    float* dst = a.S + (size_t)r.par * a.Hp + j;
+    if (partial) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(r.sum) : "memory");
+    else *dst = r.sum;
+}
+
+// One step of 16 edges for this thread's hidden unit.
+__device__ __forceinline__ void forget_step(const TcArgs& a, const Segment& sg, uint32_t taddr, int lane, int st, int j, bool j_ok,
+                                            RunSum& r, const float* sc) {
+    float g[16];
+    tmem_ld16(taddr + st * 16, g);
+    tmem_ld_wait();
+    const unsigned heads = sel4u(sg.heads, st >> 1) >> ((st & 1) * 16);
+    const int pr_sel = sel4(sg.pr, st >> 1);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        if ((heads >> e) & 1u) {   // the same in every lane: a new parent starts at this edge
+            run_flush(a, r, j, j_ok, r.runs_done == 0 && sg.cont_before);
+            r.par = __shfl_sync(0xffffffffu, pr_sel, (st & 1) * 16 + e);
+            r.sum = 0.f;
+            ++r.runs_done;
+        }
+        const float pf = sc[e * 32 + lane], ck = sc[512 + e * 32 + lane];
+        r.sum = fmaf(sigmoid_fast(pf + g[e]), ck, r.sum);
     }
 }
 
@@ -467,7 +499,7 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
                                                int total_tiles, int n_tiles, int lo, int hi, int bn, int n_leaves, int mt_leaf,
                                                int rank) {
     constexpr int TM = PAIR ? 2 * BM : BM;
-    auto tile_at = [&](int t) {
+    auto tile_at = [&](int t) {   // (not for the forget-gate GEMM, whose tiles are laid out differently)
         Tile ti = tile_of<EPI>(t, n_tiles, TM, lo, hi, bn, n_leaves, mt_leaf);
         if (PAIR) ti.row0 += rank * BM;
         return ti;
@@ -545,63 +577,47 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         }
         cp_async_wait<0>();
     } else if (EPI == EPI_F) {
-        // rows are edge slots; eight warps: this one takes the steps q = split, split + 2, ... of every tile, and the
-        // parent's forget pre-activation and the child's c of its next step arrive while it works on the current one
-        const int split = (warp - 2) >> 2;
-        float* ring = scratch + (warp - 2) * (F_RING * F_STEP_FLOATS);
+        // eight warps: lane quarter = 32 hidden units, segment = the first or the second 128 edges of the tile
+        constexpr int RING = f_ring(PAIR), STEPS = F_SEG / 16;
+        const int seg = (warp - 2) >> 2;
+        float* ring = scratch + (warp - 2) * (RING * F_STEP_FLOATS);
         const uint32_t ring_addr = smem_u32(ring);
-        const int steps = bn >> 4;
-        auto slot_rows = [&](const Tile& ti, int (&pr)[4], int (&kd)[4]) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int sl = ti.row0 + quarter * 32 + (lane >> 2) + 8 * i;
-                pr[i] = kd[i] = -1;
-                if (sl < ti.row_end) {
-                    pr[i] = a.slot_par[sl];
-                    kd[i] = a.slot_child[sl];
-                    if (a.debug && (!dbg_ok(a.meta, CHECK_PARENT_ROW, pr[i], a.n_int_bound, sl) ||
-                                    !dbg_ok(a.meta, CHECK_CHILD, kd[i], a.n_nodes, sl)))
-                        pr[i] = kd[i] = -1;
-                }
-            }
-        };
-        int f_t = t0, f_q = split, f_buf = 0;
-        Tile f_ti = tile_at(f_t);
-        int f_pr[4], f_kd[4];
-        if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
-        auto fetch_next = [&]() {
-            if (f_t < total_tiles) {
-                forget_fetch(a, f_ti, lane, f_q, f_pr, f_kd, ring_addr + (uint32_t)f_buf * (F_STEP_FLOATS * 4), ring + f_buf * F_STEP_FLOATS);
-                f_q += 2;
-                if (f_q >= steps) {
-                    f_q = split;
-                    f_t += t_step;
-                    f_ti = tile_at(f_t);
-                    if (f_t < total_tiles) slot_rows(f_ti, f_pr, f_kd);
-                }
-            }
-            cp_async_commit();
-            f_buf ^= 1;
-        };
-        fetch_next();
-        int cur = 0;
+        constexpr int TMH = PAIR ? 2 * BM : BM;   // hidden units per tile
         for (int t = t0; t < total_tiles && ok; t += t_step) {
-            const Tile ti = tile_at(t);
-            const int sl = ti.row0 + quarter * 32 + lane;   // this lane's accumulator row
-            int par = sl < ti.row_end ? a.slot_par[sl] : -1;
-            if (a.debug && par >= 0 && !dbg_ok(a.meta, CHECK_PARENT_ROW, par, a.n_int_bound, sl)) par = -1;
-            const Runs runs = runs_of(par, lane);
+            const Tile ti = tile_of<EPI>(t, n_tiles, F_EDGES, lo, hi, bn, n_leaves, mt_leaf);
+            const int j_base = ti.n_tile * TMH + rank * BM + quarter * 32, j = j_base + lane;
+            const bool j_ok = j < a.Hp;
+            const int slot0 = ti.row0 + seg * F_SEG;
+            const Segment sg = segment_of(a, slot0, ti.row_end, lane);
+            // the first steps' copies start before the accumulator is ready: they land while the tile's products run
+#pragma unroll
+            for (int st = 0; st < RING - 1; ++st) {
+                forget_fetch(a, j_base, lane, st, sel4(sg.pr, st >> 1), sel4(sg.kd, st >> 1), ring_addr + (uint32_t)st * (F_STEP_FLOATS * 4),
+                             ring + st * F_STEP_FLOATS);
+                cp_async_commit();
+            }
             if (!wait_acc(acc, acc_phase)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16);
+            const uint32_t taddr = tmem_base + (uint32_t)acc * MAX_BN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(seg * F_SEG);
+            RunSum r{0.f, -1, -1};   // the first edge of the segment always starts a run: runs_done becomes 0 there
+            int cur = 0, nxt = RING - 1;   // buffer of this step, buffer the next copies go to
 #pragma unroll 1
-            for (int q = split; q < steps; q += 2) {
-                cp_async_wait<0>();          // this step's copies have landed (they were started a step ago)
-                __syncwarp();                // ... and so have the other lanes'; the other buffer is free
-                fetch_next();
-                forget_step(a, ti, taddr, lane, q, par, runs, ring + cur * F_STEP_FLOATS);
-                cur ^= 1;
+            for (int st = 0; st < STEPS; ++st) {
+                cp_async_wait<RING - 2>();   // this step's copies have landed (they were started RING - 1 steps ago)
+                __syncwarp();                // ... and so have the other lanes'; the buffer of the step before is free
+                if (st + RING - 1 < STEPS) {
+                    const int sn = st + RING - 1;
+                    forget_fetch(a, j_base, lane, sn, sel4(sg.pr, sn >> 1), sel4(sg.kd, sn >> 1),
+                                 ring_addr + (uint32_t)nxt * (F_STEP_FLOATS * 4), ring + nxt * F_STEP_FLOATS);
+                }
+                cp_async_commit();
+                forget_step(a, sg, taddr, lane, st, j, j_ok, r, ring + cur * F_STEP_FLOATS);
+                if (++cur == RING) cur = 0;
+                if (++nxt == RING) nxt = 0;
             }
+            run_flush(a, r, j, j_ok, (r.runs_done == 0 && sg.cont_before) || sg.cont_after);
+            cp_async_wait<0>();
+            __syncwarp();                    // every lane is done with the buffers before the next tile refills them
             release_acc(acc);
             acc ^= 1;
             if (acc == 0) acc_phase ^= 1u;
@@ -730,9 +746,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         a_row_off = (EPI == EPI_LEVEL) ? -n_leaves : 0;
     }
     const int mt_leaf = is_xproj(EPI) ? (n_leaves + BM - 1) / BM : 0;
-    const int m_tiles = is_xproj(EPI) ? mt_leaf + (hi - n_leaves + BM - 1) / BM : (hi - lo + BM - 1) / BM;
-    const int n_tiles = n_total / bn;
+    // forget-gate GEMM: tiles of 256 edges x 128 hidden units, the hidden tiles of an edge tile next to each other
+    const int m_tiles = is_xproj(EPI) ? mt_leaf + (hi - n_leaves + BM - 1) / BM
+                        : EPI == EPI_F ? (hi - lo + F_EDGES - 1) / F_EDGES : (hi - lo + BM - 1) / BM;
+    const int n_tiles = EPI == EPI_F ? (a.Hp + BM - 1) / BM : n_total / bn;
     const int total_tiles = m_tiles * n_tiles;
+    constexpr int TILE_ROWS = EPI == EPI_F ? F_EDGES : BM;
 
     if (warp == 0) {
         // producer warp: lane 0 waits for the stage and issues the tile loads.  With x_gather the rows of the input
@@ -743,7 +762,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         const bool gather = is_xproj(EPI) && a.x_gather;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const Tile ti = tile_of<EPI>(t, n_tiles, BM, lo, hi, bn, n_leaves, mt_leaf);
+            const Tile ti = tile_of<EPI>(t, n_tiles, TILE_ROWS, lo, hi, bn, n_leaves, mt_leaf);
             const uint32_t tx = A_BYTES + (uint32_t)ti.bn * BK * 2;
             int rows[4] = {0, 0, 0, 0};
             if (gather) {
@@ -761,9 +780,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort);
                     if (ok) {
                         mbar_expect_tx(full, tx);
-                        if (!gather) tma_load_2d(smem_base + stage * SB, &tmA, full, kb * BK, ti.row0 + a_row_off);
+                        // forget-gate GEMM: A = 128 rows (hidden units) of U_f, B = the tile's 256 edge rows of the bf16 copy
+                        if (!gather) tma_load_2d(smem_base + stage * SB, &tmA, full, kb * BK, EPI == EPI_F ? ti.n_tile * BM : ti.row0 + a_row_off);
                         tma_load_2d(smem_base + stage * SB + A_BYTES, (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB,
-                                    full, kb * BK, is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn);
+                                    full, kb * BK, is_xproj(EPI) ? ti.n_tile * 256 : EPI == EPI_F ? ti.row0 : ti.n_tile * bn);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -783,7 +803,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const Tile ti = tile_of<EPI>(t, n_tiles, BM, lo, hi, bn, n_leaves, mt_leaf);
+                const Tile ti = tile_of<EPI>(t, n_tiles, TILE_ROWS, lo, hi, bn, n_leaves, mt_leaf);
                 const int hn = a.issuers == 2 ? ti.bn >> 1 : ti.bn;  // columns of this issuer
                 const uint32_t idesc = idesc_bf16(BM, hn);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_tempty[acc]), acc_phase ^ 1u, abort));
@@ -840,7 +860,8 @@ constexpr int STAGES2 = 6, STAGES2_LEVEL = 4;
 constexpr int STAGE2_BYTES = A_BYTES + B_BYTES_MAX / 2;
 constexpr int GEMM2_SMEM = STAGES2 * STAGE2_BYTES + 4 * EPI_STEP_FLOATS * 4 + 1024;
 constexpr int GEMM2_SMEM_LEVEL = STAGES2_LEVEL * STAGE2_BYTES + EPI_SCRATCH_BYTES + 1024;
-constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH_BYTES + 1024;
+constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH2_BYTES + 1024;
+static_assert(GEMM2_SMEM_F <= 227 * 1024 - 256, "pair forget GEMM shared memory");
 constexpr int GEMM2_SMEM_X8 = STAGES2_LEVEL * STAGE2_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;
 static_assert(GEMM2_SMEM_LEVEL <= 227 * 1024 - 256, "pair level GEMM shared memory");
 
@@ -874,8 +895,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     constexpr int TM2 = 2 * BM;
     const int mt_leaf = is_xproj(EPI) ? (n_leaves + TM2 - 1) / TM2 : 0;
+    // forget-gate GEMM: tiles of 256 edges x 256 hidden units (128 per CTA)
     const int m_tiles = is_xproj(EPI) ? mt_leaf + (hi - n_leaves + TM2 - 1) / TM2 : (hi - lo + TM2 - 1) / TM2;
-    const int n_tiles = n_total / bn;
+    const int n_tiles = EPI == EPI_F ? (a.Hp + TM2 - 1) / TM2 : n_total / bn;
     const int total_tiles = m_tiles * n_tiles;
 
     if (threadIdx.x == 0) {
@@ -926,9 +948,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort);
                     if (ok) {
                         if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[stage]), tx);
-                        if (!gather) tma_load_2d_pair(smem_base + stage * STAGE2_BYTES, &tmA, full_leader, kb * BK, my_row0 + a_row_off);
+                        // forget-gate GEMM: A = this CTA's 128 of the tile's 256 hidden units of U_f, B = its half of the edges
+                        if (!gather) tma_load_2d_pair(smem_base + stage * STAGE2_BYTES, &tmA, full_leader, kb * BK,
+                                                      EPI == EPI_F ? ti.n_tile * TM2 + (int)rank * BM : my_row0 + a_row_off);
                         // this CTA's half of the B tile's rows (the MMA reads rows 0.. from CTA 0, the rest from CTA 1)
-                        const int n_base = is_xproj(EPI) ? ti.n_tile * 256 : ti.n_tile * bn;
+                        const int n_base = is_xproj(EPI) ? ti.n_tile * 256 : EPI == EPI_F ? ti.row0 : ti.n_tile * bn;
                         const CUtensorMap* tb = (is_xproj(EPI) && ti.bn == 192) ? &tmB_leaf : &tmB;
                         tma_load_2d_pair(smem_base + stage * STAGE2_BYTES + A_BYTES, tb, full_leader, kb * BK,
                                          n_base + (int)rank * half_bn);
@@ -1456,8 +1480,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     const bool big = !use_small && (long long)N >= 2LL * BM * n_sm;
     const bool pair_x = big && (tune.pair_mask & 1), pair_l = big && (tune.pair_mask & 2), pair_f = big && (tune.pair_mask & 4);
     const uint32_t bdiv = pair_x ? 2 : 1, bdiv_l = pair_l ? 2 : 1;
-    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmUf, tmUfH, tmP, tmHBs;
-    const int bnf = g_bn(Hp);
+    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmHBh, tmUf, tmP, tmHBs;
     // W is read through a full box and a leaf box (i, o, u blocks only)
     bool ok = (a.x_gather ? make_tmap(&tmX, fa.x, n, (uint64_t)D, (uint64_t)fa.ldx, 1)    // one-row boxes for the gathers
                           : make_tmap(&tmX, w.xb, n, (uint64_t)D, (uint64_t)Dp, BM)) &&
@@ -1466,9 +1489,9 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     if (ok && !use_small)   // the per-level launches read their operands through five more maps
         ok = make_tmap(&tmHS, w.hs, ni, (uint64_t)Hp, (uint64_t)Hp, BM) &&
              make_tmap(&tmUiou, pk + L.off_Uiou, (uint64_t)3 * Hp, (uint64_t)Hp, (uint64_t)Hp, 192 / bdiv_l) &&
-             make_tmap(&tmHB, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, BM) &&
-             make_tmap(&tmUf, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bnf) &&
-             make_tmap(&tmUfH, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, (uint32_t)bnf / 2);
+             make_tmap(&tmHB, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, F_EDGES) &&        // forget-gate GEMM: B, a tile's 256 edge rows
+             make_tmap(&tmHBh, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, F_EDGES / 2) &&   // ... half of them per CTA of a pair
+             make_tmap(&tmUf, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, BM);   // ... A, 128 hidden units
     ok = ok && make_tmap_f32(&tmP, w.P, ni, (uint64_t)4 * Hp, (uint64_t)4 * Hp) &&
          make_tmap(&tmHBs, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, 32);  // store boxes: 64 columns x one warp's 32 rows
     if (!ok) return JDB_ERR_UNSUPPORTED;
@@ -1496,13 +1519,16 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     // one GEMM launch: a lone-CTA grid, or a grid of CTA pairs (clusters of 2) for launches with many tiles
     auto launch = [&](int epi, const CUtensorMap& tA, const CUtensorMap& tB_full, const CUtensorMap& tBl, long long rows_bound,
                       int level, int bn, int n_total, int kblocks) -> jdb_status {
-        const int n_tiles = n_total / bn;
+        // tiles along the second dimension: N tiles of the weights, or (forget-gate GEMM) tiles of hidden units
+        const int n_tiles = epi == EPI_F ? (Hp + BM - 1) / BM : n_total / bn;
+        const int n_tiles2 = epi == EPI_F ? (Hp + 2 * BM - 1) / (2 * BM) : n_tiles;
         // the forget-gate GEMM decides launch by launch: pairs pay off from about 32 tiles per pair on
-        const long long tiles2 = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles;
+        const long long tiles2 = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles2;
         const bool pair = is_xproj(epi) ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_f && tiles2 >= 32LL * (n_sm / 2));
-        const CUtensorMap& tB = (epi == EPI_F && pair) ? tmUfH : tB_full;
+        const CUtensorMap& tB = (epi == EPI_F && pair) ? tmHBh : tB_full;
         if (!pair) {
-            const int grid = gemm_grid(rows_bound, n_tiles);
+            const long long lone_tiles = epi == EPI_F ? (rows_bound + F_EDGES - 1) / F_EDGES * n_tiles : 0;
+            const int grid = epi == EPI_F ? (int)(lone_tiles < n_sm ? (lone_tiles > 0 ? lone_tiles : 1) : n_sm) : gemm_grid(rows_bound, n_tiles);
             if (epi == EPI_XPROJ) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_STORE, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
             else if (epi == EPI_XPROJ8) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_XPROJ8>, dim3(grid), dim3(GEMMF_THREADS), GEMM_SMEM_X8, st, tA, tB, tBl, tmP, tmHBs, af, level, bn, n_total, kblocks));
             else if (epi == EPI_LEVEL) JDB_CUDA_TRY(launch_behind(tune.pdl, gemm_tc_kernel<EPI_LEVEL>, dim3(grid), dim3(GEMM1_THREADS), GEMM_SMEM_LEVEL, st, tA, tB, tBl, tmP, tmHBs, a, level, bn, n_total, kblocks));
@@ -1563,7 +1589,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         const int cs_blocks = (int)((ni + 7) / 8 < (size_t)n_sm * 8 ? (ni + 7) / 8 : (size_t)n_sm * 8);
         for (int level = 1; level < n_levels; ++level) {
             JDB_CUDA_TRY(launch_behind(tune.pdl, childsum_kernel, dim3(cs_blocks), dim3(256), 0, st, a, level));
-            if ((ls = launch(EPI_F, tmHB, tmUf, tmUf, (long long)fa.n_edges, level, bnf, Hp, kh)) != JDB_OK) return ls;
+            if ((ls = launch(EPI_F, tmUf, tmHB, tmHB, (long long)fa.n_edges, level, F_EDGES, F_EDGES, kh)) != JDB_OK) return ls;
             if ((ls = launch(EPI_LEVEL, tmHS, tmUiou, tmUiou, (long long)ni, level, 192, 3 * Hp, kh)) != JDB_OK) return ls;
         }
         JDB_CUDA_TRY(cudaGetLastError());
