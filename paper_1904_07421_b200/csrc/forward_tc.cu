@@ -459,11 +459,11 @@ struct RunSum {
     float sum;
     int par, runs_done;
 };
-__device__ __forceinline__ void run_flush(const TcArgs& a, const RunSum& r, int j, bool j_ok, bool partial) {
-    if (r.par < 0 || !j_ok) return;
-    float* dst = a.S + (size_t)r.par * a.Hp + j;
-    if (partial) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(r.sum) : "memory");
-    else *dst = r.sum;
+__device__ __forceinline__ void run_flush(float* S, int Hp, float sum, int par, int j, bool j_ok, bool partial) {
+    if (par < 0 || !j_ok) return;
+    float* dst = S + (size_t)par * Hp + j;
+    if (partial) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(sum) : "memory");
+    else *dst = sum;
 }
 
 // One step of 16 edges for this thread's hidden unit.
@@ -474,16 +474,20 @@ __device__ __forceinline__ void forget_step(const TcArgs& a, const Segment& sg, 
     tmem_ld_wait();
     const unsigned heads = sel4u(sg.heads, st >> 1) >> ((st & 1) * 16);
     const int pr_sel = sel4(sg.pr, st >> 1);
+    // first all sixteen products, free of branches, so that their chains of dependent instructions (shared-memory
+    // load, add, tanh, multiply) overlap; then the cheap serial part, which alone depends on where parents change
+    float fc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) fc[e] = sigmoid_fast(sc[e * 32 + lane] + g[e]) * sc[512 + e * 32 + lane];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
         if ((heads >> e) & 1u) {   // the same in every lane: a new parent starts at this edge
-            run_flush(a, r, j, j_ok, r.runs_done == 0 && sg.cont_before);
+            run_flush(a.S, a.Hp, r.sum, r.par, j, j_ok, r.runs_done == 0 && sg.cont_before);
             r.par = __shfl_sync(0xffffffffu, pr_sel, (st & 1) * 16 + e);
             r.sum = 0.f;
             ++r.runs_done;
         }
-        const float pf = sc[e * 32 + lane], ck = sc[512 + e * 32 + lane];
-        r.sum = fmaf(sigmoid_fast(pf + g[e]), ck, r.sum);
+        r.sum += fc[e];
     }
 }
 
@@ -615,7 +619,7 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
                 if (++cur == RING) cur = 0;
                 if (++nxt == RING) nxt = 0;
             }
-            run_flush(a, r, j, j_ok, (r.runs_done == 0 && sg.cont_before) || sg.cont_after);
+            run_flush(a.S, a.Hp, r.sum, r.par, j, j_ok, (r.runs_done == 0 && sg.cont_before) || sg.cont_after);
             cp_async_wait<0>();
             __syncwarp();                    // every lane is done with the buffers before the next tile refills them
             release_acc(acc);
