@@ -244,12 +244,16 @@ def level_loop_bytes(w: wl.Workload, n_leaves: int):
 # of the named kernels on the named workload, from the captures summarised under profiles/; None where a kernel has
 # changed since its counters were taken.
 MEASURED_TRAFFIC = {
-    ("small_levels_kernel", 2): None,
-    ("small_levels_kernel", 4): None,
-    ("small_levels_f32_kernel", 1): None,
-    ("gemm_tc_kernel<EPI_XPROJ>", 5): None,
-    ("per-level loop", 3): None,
-    ("per-level loop", 5): None,
+    ("small_levels_f32_kernel", 1): 2231040,            # whole workload captured, one launch
+    ("small_levels_kernel", 2): 5665792,                # whole workload captured, one launch
+    ("small_levels_kernel", 4): 896706560,              # whole workload captured, one launch
+    # per-level loop = all childsum_kernel, gemm_tc_kernel<EPI_F> and gemm_tc_kernel<EPI_LEVEL> launches of one step
+    ("per-level loop", 3): 1656050000,                  # whole workload captured (12 levels, 36 launches)
+    # captured on 8192 of the 65536 trees (194583 nodes: 2765 MB) and scaled by the node count: every row is read and
+    # written a fixed number of times, so traffic grows in proportion
+    ("per-level loop", 5): int(2765.0e6 * (1571637 / 194583)),
+    # input projection of workload 5, four-warp kernel: captured on the same 8192 trees (408.6 + 2036.3 MB), scaled
+    ("gemm_tc_kernel<EPI_XPROJ>", 5): int((408579072 + 2036310000) * (1571637 / 194583)),
 }
 
 

@@ -1583,10 +1583,12 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         edge_fill_kernel<<<(int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16), 256, 0, st>>>(a, w.block_sum);
         JDB_CUDA_TRY(cudaGetLastError());
     }
-    // eight epilogue warps where the bf16 copy of h goes out row by row anyway (child order) and the forest is large
-    // enough for the epilogue to matter; the small forests of the cooperative loop keep the four-warp kernel, whose
-    // leaf tiles leave as one TMA box per warp
-    const int xepi = (!use_small && !tune.issuers2_requested) ? EPI_XPROJ8 : EPI_XPROJ;
+    // Eight epilogue warps where the bf16 copy of h goes out row by row anyway (child order) and K is short: with at
+    // most eight K blocks per tile the epilogue weighs more than the pipeline stage the eight step buffers cost
+    // (D = 512: 0.47 -> 0.44 ms on 143 k nodes); at sixteen K blocks the four-stage kernel is ahead (D = 1024: 1.16 vs
+    // 1.22 ms on 195 k nodes).  The small forests of the cooperative loop keep the four-warp kernel, whose leaf tiles
+    // leave as one TMA box per warp.
+    const int xepi = (!use_small && !tune.issuers2_requested && kd <= 8) ? EPI_XPROJ8 : EPI_XPROJ;
     if ((ls = launch(xepi, tmX, tmW, tmWl, (long long)N + 2 * BM, 0, 256, 4 * Hp, kd)) != JDB_OK) return ls;
     if (fa.ev_xproj_done) JDB_CUDA_TRY(cudaEventRecord(fa.ev_xproj_done, st));
     if (!use_small) {
