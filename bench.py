@@ -252,8 +252,9 @@ MEASURED_TRAFFIC = {
     # captured on 8192 of the 65536 trees (194583 nodes: 2765 MB) and scaled by the node count: every row is read and
     # written a fixed number of times, so traffic grows in proportion
     ("per-level loop", 5): int(2765.0e6 * (1571637 / 194583)),
-    # input projection of workload 5, four-warp kernel: captured on the same 8192 trees (408.6 + 2036.3 MB), scaled
-    ("gemm_tc_kernel<EPI_XPROJ>", 5): int((408579072 + 2036310000) * (1571637 / 194583)),
+    # input projection of workload 5 (four-warp kernel, rows of the bf16 copy to their slots): one launch captured on the
+    # same 8192 trees (408.59 MB read, 2034.67 MB written), scaled
+    ("gemm_tc_kernel<EPI_XPROJ>", 5): int(2443266816 * (1571637 / 194583)),
 }
 
 
@@ -427,6 +428,36 @@ def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device
     return ms, h2d, d2h
 
 
+def time_head(w: wl.Workload, job: GpuJob, flush, pk, Hs: int = 50, K: int = 5, reps: int = 10):
+    """The relatedness head over the forest's root states (pairs of consecutive trees): time per call and the
+    fraction of the copy bandwidth its algorithmic bytes (two root rows per pair) reach.  Not part of `value`."""
+    torch, jdb = job.torch, job.jdb
+    rng = np.random.default_rng(7)
+    H = w.H
+    dev = job.h.device
+    mk = lambda *shape: torch.from_numpy(rng.uniform(-0.3, 0.3, shape).astype(np.float32)).to(dev)
+    Wx, Wp, bh, Wq, bq = mk(Hs, H), mk(Hs, H), mk(Hs), mk(K, Hs), mk(K)
+    roots = torch.from_numpy(w.forest.roots.astype(np.int32)).to(dev)
+    left, right = roots[0::2].contiguous(), roots[1::2].contiguous()
+    n_pairs = int(min(left.numel(), right.numel()))
+    left, right = left[:n_pairs], right[:n_pairs]
+    if n_pairs == 0:
+        return None
+    ms = []
+    for _ in range(reps + 3):
+        flush.add_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        jdb.jdb_relatedness_head(job.h, left, right, Wx, Wp, bh, Wq, bq, want_p=False)
+        e1.record()
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    t = statistics.median(ms[3:])
+    bytes_ = n_pairs * 2 * H * 4
+    return {"pairs": n_pairs, "ms": t, "pairs_per_s": n_pairs / (t * 1e-3), "algorithmic_bytes": bytes_,
+            "frac_of_hbm_peak": bytes_ / (t * 1e-3) / 1e9 / pk["hbm_gbs"], "head_hidden": Hs, "classes": K}
+
+
 def rank_workload(config: int, rank: int, n_trees=None) -> wl.Workload:
     """Every rank draws its own forest of the workload's shape (weak scaling over independent trees)."""
     return wl.make_workload(config, n_trees=n_trees, seed=None if rank == 0 else wl.BASE_SEED + config + 1000 * rank)
@@ -510,6 +541,9 @@ def run_gpu(args):
     n_levels_main, launches_main = job.n_levels, job.launches_per_step()
     precision_main, packed_main = job.precision, job.packed
 
+    # the workload's scoring step (Section 5: relatedness of sentence pairs): consecutive trees form a pair
+    head = time_head(w, job, flush, pk)
+
     # end to end from pinned host buffers through the host entry point (the resident buffers are released first)
     job.plan = None
     job.x = job.h = job.c = job.fws = job.sws = None
@@ -556,6 +590,7 @@ def run_gpu(args):
             "roofline": roofline,
             "path_frac_of_roofline": path_frac,
             "phases": phases_out,
+            "relatedness_head": head,
             "batching_ratio": f.n_nodes / max(n_levels_main, 1),   # cells evaluated per batched step: Section 3's batching ratio at cell granularity
             "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample,
                              "parallel_over_trees": cpu_par},

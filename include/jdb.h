@@ -222,6 +222,23 @@ jdb_status jdb_sched_status(const jdb_sched *sched, int32_t *n_levels_out, int32
  * The companion of the depth-ordered execution of Section 4.2 for callers that assemble schedules themselves. */
 jdb_status jdb_debug_report(const jdb_sched *sched, int32_t out[4], void *stream);
 
+/* ---- relatedness head (the scoring function of the workload of Section 5) --------------------- */
+
+/* Scores pairs of trees from the states of their roots, with the head of the Tree-LSTM model the paper cites:
+ *     h_s = sig(W_x (h_L * h_R) + W_+ |h_L - h_R| + b_h);  p = softmax(W_p h_s + b_p);  y = sum_k k p_k, k = 1..K.
+ * h        [n_nodes, H] fp32 with leading dimension ldh: the h output of jdb_treelstm_forward.
+ * left, right  [n_pairs] node ids of the two roots of every pair.
+ * Wx, Wp   [Hs, H] row-major (the weights of the product and of the difference features), bh [Hs];
+ * Wq [K, Hs], bq [K]; K <= 32; 4 (2 H + Hs) floats must fit 48 KB of shared memory (H up to about 1500), else
+ * JDB_ERR_UNSUPPORTED.
+ * y        [n_pairs] fp32 out;  p [n_pairs, K] fp32 out, may be NULL.
+ * bad_flag one int32 on the device, set to 1 if a root id lies outside 0 .. n_nodes-1 (that pair is skipped), else 0.
+ * All pointers are device pointers.  Asynchronous on `stream`; allocates nothing. */
+jdb_status jdb_relatedness_head(const float *h, int64_t ldh, int32_t n_nodes, const int32_t *left, const int32_t *right,
+                                int32_t n_pairs, const float *Wx, const float *Wp, const float *bh, const float *Wq,
+                                const float *bq, int32_t H, int32_t Hs, int32_t K, float *y, float *p, int32_t *bad_flag,
+                                void *stream);
+
 /* ---- one call from host buffers (what a user without device arrays calls) -------------------- */
 
 /* Device scratch needed by jdb_treelstm_forward_host (CSR, x, schedule, h, c and both workspaces). */

@@ -28,7 +28,7 @@ EXPORTS = [
     "jdb_status_string", "jdb_last_cuda_error", "jdb_schedule_workspace_bytes", "jdb_schedule",
     "jdb_schedule_async", "jdb_schedule_static", "jdb_packed_weights_bytes", "jdb_pack_weights", "jdb_forward_workspace_bytes",
     "jdb_treelstm_forward", "jdb_sched_status", "jdb_debug_report", "jdb_forward_host_workspace_bytes",
-    "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts",
+    "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts", "jdb_relatedness_head",
 ]
 
 
@@ -101,6 +101,8 @@ def lib():
     L.jdb_launch_counts_workspace_bytes.argtypes = [i32]
     L.jdb_launch_counts.restype = C.c_int
     L.jdb_launch_counts.argtypes = [C.POINTER(CForest), C.POINTER(CSched), C.POINTER(CLaunchStats), vp, sz, vp]
+    L.jdb_relatedness_head.restype = C.c_int
+    L.jdb_relatedness_head.argtypes = [vp, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
     L.jdb_forward_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
     L.jdb_treelstm_forward_host.restype = C.c_int
@@ -273,6 +275,25 @@ def jdb_launch_counts(forest: Forest, sched: Schedule, ws: Optional[torch.Tensor
     if st != OK:
         raise JdbError(st, "jdb_launch_counts")
     return out.cells_unbatched, out.cells_batched, out.ops_unbatched, out.ops_batched, out.n_levels
+
+
+def jdb_relatedness_head(h: torch.Tensor, left: torch.Tensor, right: torch.Tensor, Wx: torch.Tensor, Wp: torch.Tensor,
+                         bh: torch.Tensor, Wq: torch.Tensor, bq: torch.Tensor, stream=None, want_p: bool = True):
+    """(y [P], p [P, K]) for pairs of root states taken from h [n, >= H] (fp32, row stride h.stride(0))."""
+    Hs, H = Wx.shape
+    K = Wq.shape[0]
+    P = int(left.numel())
+    dev = h.device
+    Wx, Wp, bh, Wq, bq = (t.to(torch.float32).contiguous() for t in (Wx, Wp, bh, Wq, bq))
+    left, right = left.to(torch.int32).contiguous(), right.to(torch.int32).contiguous()
+    y = torch.empty(max(P, 1), dtype=torch.float32, device=dev)
+    p = torch.empty((max(P, 1), K), dtype=torch.float32, device=dev) if want_p else None
+    bad = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().jdb_relatedness_head(_ptr(h), h.stride(0), h.shape[0], _ptr(left), _ptr(right), P, _ptr(Wx), _ptr(Wp), _ptr(bh),
+                                    _ptr(Wq), _ptr(bq), H, Hs, K, _ptr(y), _ptr(p), _ptr(bad), _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_relatedness_head")
+    return y[:P], (p[:P] if want_p else None), bad
 
 
 def jdb_debug_report(sched: Schedule, stream=None):
