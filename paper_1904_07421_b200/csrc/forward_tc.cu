@@ -1371,12 +1371,6 @@ cudaError_t launch_behind(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-int g_bn(int Hp) {  // N tile of the U_f GEMM: the largest multiple of 64 up to 256 that divides Hp
-    for (int m = 4; m >= 1; --m)
-        if (Hp % (64 * m) == 0) return 64 * m;
-    return 64;
-}
-
 }  // namespace
 
 TcPackLayout tc_pack_layout(int32_t D, int32_t H) {
