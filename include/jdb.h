@@ -56,7 +56,7 @@ enum {
 };
 
 /* jdb_opts.tuning: 0 takes the library's defaults (the measured best, which the environment variables JDB_GEMM_PAIR,
- * JDB_GEMM_ISSUERS, JDB_PDL, JDB_P_TMA and JDB_GATHER_X may change, read at every call).  With JDB_TUNE_SET the other bits
+ * JDB_GEMM_ISSUERS, JDB_PDL, JDB_P_TMA, JDB_GATHER_X and JDB_TREE_GROUPS may change, read at every call).  With JDB_TUNE_SET the other bits
  * replace those defaults for this call; every combination computes the same values. */
 enum {
     JDB_TUNE_SET = 1,
@@ -66,8 +66,12 @@ enum {
     JDB_TUNE_TWO_ISSUERS = 16,  /* two MMA-issuing warps per lone CTA, half of the tile's columns each               */
     JDB_TUNE_NO_PDL = 32,       /* ordinary launches instead of programmatic dependent launches                      */
     JDB_TUNE_PLAIN_STORES = 64, /* level-ordered outputs through the load/store units instead of TMA stores           */
-    JDB_TUNE_GATHER_X = 128     /* bf16 x with 16-byte aligned rows is read in place by the input projection (TMA row
+    JDB_TUNE_GATHER_X = 128,    /* bf16 x with 16-byte aligned rows is read in place by the input projection (TMA row
                                    gathers keyed by perm) instead of being laid out in level order first; slower      */
+    JDB_TUNE_TREE_GROUPS = 256  /* cooperative level loop (JDB_BF16, H <= 192): partition the forest by tree over the groups
+                                   of CTAs, which then synchronise inside a group only instead of ending every level in
+                                   a barrier over the whole grid (needs a schedule from jdb_schedule; not faster on the
+                                   workloads measured, so off by default)                                                */
 };
 
 #define JDB_META_INTS 16 /* size of jdb_sched.meta in int32 */

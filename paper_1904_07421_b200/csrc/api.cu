@@ -210,6 +210,7 @@ jdb_status jdb_treelstm_forward(const jdb_forest* forest, const jdb_sched* sched
     a.ev_levels_done = (cudaEvent_t)opts->ev_levels_done;
     a.trace = (unsigned long long*)opts->trace;
     a.trace_cap = opts->trace ? opts->trace_cap : 0;
+    a.depth = sched->depth;
     a.tuning = opts->tuning;
     a.debug = (opts->flags & JDB_FLAG_DEBUG_CHECKS) ? 1 : 0;
 

@@ -125,6 +125,7 @@ struct ForwardArgs {
     cudaEvent_t ev_begin, ev_xproj_done, ev_levels_done;  // optional timing hooks (null = none)
     unsigned long long* trace;                             // optional level trace (null = none)
     long long trace_cap;
+    const int32_t* depth;                                  // jdb_sched.depth (may be null)
     int32_t tuning;                                        // jdb_opts.tuning
     int32_t debug;                                         // 1: JDB_FLAG_DEBUG_CHECKS
 };
@@ -150,12 +151,28 @@ size_t forward_tc_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D,
 jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int n_levels, int n_internal_bound,
                               void* ws, bool use_small, uint64_t timeout_ns, cudaStream_t st);
 
+// ---- partition.cu -----------------------------------------------------------------------------
+// Tree partition for the cooperative level loop: nodes ordered by (depth, group) and the offsets of every
+// (depth, group) range; gbar holds one barrier counter per group (zeroed by partition_enqueue).
+constexpr long long PARTITION_TABLE_MAX = 1 << 20;   // (depth, group) pairs the offset table can hold
+constexpr int PARTITION_MAX_GROUPS = 1024;
+struct Partition {
+    const int32_t* gperm;  // [n_nodes]
+    const int32_t* goff;   // [n_levels * G + 1]
+    int32_t* gbar;         // [G]
+    int32_t G;             // 0: no partition (levels are separated by grid-wide barriers)
+};
+size_t partition_ws_bytes(int32_t n_nodes);
+jdb_status partition_enqueue(const ForwardArgs& fa, const int32_t* depth, int n_levels, int G, void* ws, Partition* out, cudaStream_t st);
+
 // ---- forward_small.cu -------------------------------------------------------------------------
 bool small_levels_supported(int32_t H);
 // hb: bf16 copy of h, [n_nodes][Hp], rows in level order (leaf rows filled by the input projection);
 // inv: position of every node in level order
+// part: tree partition (G > 0: every group of CTAs walks its own trees, synchronising inside the group only), or G = 0
+int small_levels_groups(int32_t H, int n_internal_bound);   // CTA groups the cooperative launch will have (0: unsupported)
 jdb_status small_levels_enqueue(const ForwardArgs& fa, const void* packed_tc, const float* P, void* hb, const int32_t* inv,
-                                int n_internal_bound, int first_level, uint64_t timeout_ns, cudaStream_t st);
+                                int n_internal_bound, int first_level, uint64_t timeout_ns, const Partition& part, cudaStream_t st);
 
 // ---- forward_small_f32.cu ---------------------------------------------------------------------
 // the fp32 level loop as one cooperative launch with resident weight slices (H <= 192); reads fa.P as written by

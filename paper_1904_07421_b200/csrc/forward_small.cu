@@ -65,6 +65,11 @@ struct SmallArgs {
     int32_t first_level;  // levels below it were evaluated by launches of their own
     int32_t n_nodes, n_edges;
     int32_t debug;        // check every index against its array before following it
+    // tree partition (G > 0: the launch has exactly G groups; each walks its own trees and synchronises inside the group)
+    const int32_t* gperm;
+    const int32_t* goff;
+    int32_t* gbar;
+    int32_t G;
     unsigned long long* trace;
     long long trace_cap;
 };
@@ -136,7 +141,8 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
         if (mt > 1) atomicMax(&s_max_tiles, mt);
     }
     __syncthreads();
-    const int active_grp = min(n_grp, s_max_tiles);
+    const bool grouped = a.G > 0;   // every group takes part: it owns trees of its own
+    const int active_grp = grouped ? n_grp : min(n_grp, s_max_tiles);
     const unsigned active_ctas = (unsigned)(active_grp * a.n_slices);
     if (grp >= active_grp) alive = false;
 
@@ -144,13 +150,13 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
         // ================= description warps: run ahead of the arithmetic by up to two passes =================
         if (alive) {
             DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, a.inv, a.first_level, n_levels, grp, n_grp, active_grp, nt_max,
-                           a.meta, a.n_nodes, a.n_edges, a.debug};
-            describe_passes(d, ring, ET, abort, tid - MAIN_THREADS, [&](int pos0, int m, int tcount, int tm) {
+                           a.meta, a.n_nodes, a.n_edges, a.debug, a.gperm, a.goff, a.G, n_leaves};
+            describe_passes(d, ring, ET, abort, tid - MAIN_THREADS, [&](const PassSlot& S, int m, int tcount, int tm) {
                 // forget slices of the tile's input projection, for this CTA's hidden units (parity selects the buffer)
                 float* dst = pfs + (tcount & 1) * (NT_MAX * PF_LD);
                 for (int task = tm; task < m * (SBJ / 4); task += META_THREADS) {
                     const int r = task >> 3, q = task & 7;
-                    cp_async16(smem_u32(dst + r * PF_LD + 4 * q), a.P + ((size_t)(pos0 + r - n_leaves) * 4 + 3) * Hp + j0 + 4 * q);
+                    cp_async16(smem_u32(dst + r * PF_LD + 4 * q), a.P + ((size_t)S.prow[r] * 4 + 3) * Hp + j0 + 4 * q);
                 }
             });
         }
@@ -166,14 +172,17 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(gate * SBJ);
         uint32_t mma_phase = 0;
         int k = 0, tcount = 0;
+        const DescribeArgs dm{a.child_ptr, a.child_idx, a.level_ptr, a.perm, a.inv, a.first_level, n_levels, grp, n_grp, active_grp, nt_max,
+                              a.meta, a.n_nodes, a.n_edges, a.debug, a.gperm, a.goff, a.G, n_leaves};
         for (int level = a.first_level; level < n_levels && alive; ++level) {
             int lo, hi;
-            checked_level(a.level_ptr, level, a.n_nodes, a.meta, a.debug, lo, hi);
-            const int nt = tile_nodes(hi - lo, nt_max, n_grp);
+            group_level(dm, level, lo, hi);   // the same ranges and tiles as the description warps walk
+            const int nt = tile_nodes(hi - lo, nt_max, grouped ? 1 : n_grp);
             const int tiles = (hi - lo + nt - 1) / nt;
             stamp(level, 0, true);
-            for (int tile = grp; tile < tiles && alive; tile += active_grp, ++tcount) {
-                const bool first = tile == grp;
+            const int tile0 = grouped ? 0 : grp, tile_step = grouped ? 1 : active_grp;
+            for (int tile = tile0; tile < tiles && alive; tile += tile_step, ++tcount) {
+                const bool first = tile == tile0;
                 float zi[RPT], zo[RPT], zu[RPT], sfc[RPT];  // running sums of this thread's (row, hidden unit) pairs
 #pragma unroll
                 for (int i = 0; i < RPT; ++i) zi[i] = zo[i] = zu[i] = sfc[i] = 0.f;
@@ -183,7 +192,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                     const bool good = mbar_wait_warp(smem_u32(&ring.bar_full[s]), (uint32_t)((k >> 1) & 1), abort);
                     if (!good) *abort = 1;
                     const PassSlot& S = ring.slot[s];
-                    const int pos0 = S.pos0, m = S.m, ne = S.ne, et0 = S.et0;
+                    const int m = S.m, ne = S.ne, et0 = S.et0;
                     const int nc = good ? min(ET, ne - et0) : 0;
                     last = !good || et0 + ET >= ne;
                     stamp(level, 1, first && et0 == 0);
@@ -223,7 +232,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                         const int r = warp + MAIN_WARPS * i;
                         pi[i] = po[i] = pu[i] = 0.f;
                         if (last && r < m) {
-                            const float* prow = a.P + (size_t)(pos0 + r - n_leaves) * 4 * Hp + j0 + lane;
+                            const float* prow = a.P + (size_t)S.prow[r] * 4 * Hp + j0 + lane;
                             pi[i] = __ldg(prow);
                             po[i] = __ldg(prow + Hp);
                             pu[i] = __ldg(prow + 2 * Hp);
@@ -292,7 +301,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
                             const unsigned mine = (unsigned)__bfloat16_as_ushort(hb16);
                             const unsigned next = __shfl_down_sync(0xffffffffu, mine, 1);
                             if ((lane & 1) == 0)
-                                *reinterpret_cast<uint32_t*>(a.hb + (size_t)(pos0 + r) * Hp + j0 + lane) = mine | (next << 16);
+                                *reinterpret_cast<uint32_t*>(a.hb + (size_t)(S.prow[r] + n_leaves) * Hp + j0 + lane) = mine | (next << 16);
                         }
                     }
                     named_bar(BAR_MAIN, MAIN_THREADS);  // exchange buffer, operand and slot are free again
@@ -303,7 +312,10 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
             }
             if (!alive) break;
             if (level + 1 < n_levels) {
-                if (!main_grid_barrier(a.meta, (unsigned)(level - a.first_level + 1) * active_ctas, a.timeout_ns, abort, tid)) alive = false;
+                // all participating CTAs meet, or (tree partition) the CTAs of this group only
+                int32_t* counter = grouped ? &a.gbar[grp] : &a.meta[META_BARRIER];
+                const unsigned per_level = grouped ? (unsigned)a.n_slices : active_ctas;
+                if (!main_grid_barrier(a.meta, counter, (unsigned)(level - a.first_level + 1) * per_level, a.timeout_ns, abort, tid)) alive = false;
             }
             stamp(level, 7, true);
         }
@@ -319,14 +331,24 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_kernel(SmallArgs a) 
 
 bool small_levels_supported(int32_t H) { return H <= SMAX_KB * 64; }
 
+int small_levels_groups(int32_t H, int n_internal_bound) {
+    if (!small_levels_supported(H)) return 0;
+    DevInfo* di = dev_info();
+    if (!di) return 0;
+    const int n_slices = (H + SBJ - 1) / SBJ;
+    int groups = di->n_sm / n_slices;  // one CTA per SM: the kernel uses most of an SM's shared memory
+    const int max_tiles = ceil_div(n_internal_bound > 0 ? n_internal_bound : 1, 32);
+    if (groups > max_tiles) groups = max_tiles;
+    return groups;
+}
+
 jdb_status small_levels_enqueue(const ForwardArgs& fa, const void* packed_tc, const float* P, void* hb, const int32_t* inv,
-                                int n_internal_bound, int first_level, uint64_t timeout_ns, cudaStream_t st) {
+                                int n_internal_bound, int first_level, uint64_t timeout_ns, const Partition& part, cudaStream_t st) {
     const int H = fa.H;
     TcPackLayout L = tc_pack_layout(fa.D, H);
     if (!small_levels_supported(H)) return JDB_ERR_UNSUPPORTED;
     DevInfo* di = dev_info();
     if (!di) return JDB_ERR_CUDA;
-    const int n_sm = di->n_sm;
     if (!(di->attr_mask & ATTR_SMALL_LEVELS)) {
         JDB_CUDA_TRY(cudaFuncSetAttribute(small_levels_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMALL_SMEM));
         di->attr_mask |= ATTR_SMALL_LEVELS;
@@ -355,10 +377,10 @@ jdb_status small_levels_enqueue(const ForwardArgs& fa, const void* packed_tc, co
 
     a.n_nodes = fa.n_nodes; a.n_edges = fa.n_edges;
     a.debug = fa.debug;
-    int groups = n_sm / a.n_slices;  // one CTA per SM: the kernel uses most of an SM's shared memory
-    const int max_tiles = ceil_div(n_internal_bound > 0 ? n_internal_bound : 1, 32);
-    if (groups > max_tiles) groups = max_tiles;
+    const int groups = small_levels_groups(H, n_internal_bound);
     if (groups < 1) return JDB_ERR_UNSUPPORTED;
+    if (part.G > 0 && part.G != groups) return JDB_ERR_INVALID_ARG;   // the partition was made for another launch shape
+    a.gperm = part.gperm; a.goff = part.goff; a.gbar = part.gbar; a.G = part.G;
     void* params[] = {&a};
     JDB_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)small_levels_kernel, dim3(groups * a.n_slices), dim3(STHREADS), params,
                                              SMALL_SMEM, st));

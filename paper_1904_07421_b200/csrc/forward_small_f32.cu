@@ -127,13 +127,13 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
         // ================= description warps =================
         if (alive) {
             DescribeArgs d{a.child_ptr, a.child_idx, a.level_ptr, a.perm, nullptr, 1, n_levels, grp, n_grp, active_grp, FNT_RULE,
-                           a.meta, a.n_nodes, a.n_edges, a.debug};
-            describe_passes(d, ring, FET, abort, tid - MAIN_THREADS, [&](int pos0, int m, int tcount, int tm) {
+                           a.meta, a.n_nodes, a.n_edges, a.debug, nullptr, nullptr, 0, n_leaves};
+            describe_passes(d, ring, FET, abort, tid - MAIN_THREADS, [&](const PassSlot& S, int m, int tcount, int tm) {
                 // the tile's input projection for this CTA's hidden units (parity selects the buffer)
                 float4* dst = pst + (tcount & 1) * (FNT * SBJ);
                 for (int task = tm; task < m * SBJ; task += META_THREADS) {
                     const int r = task >> 5, jj = task & 31;
-                    if (j0 + jj < H) cp_async16(smem_u32(dst + r * SBJ + jj), a.P4 + (size_t)(pos0 + r - n_leaves) * H + j0 + jj);
+                    if (j0 + jj < H) cp_async16(smem_u32(dst + r * SBJ + jj), a.P4 + (size_t)S.prow[r] * H + j0 + jj);
                     else dst[r * SBJ + jj] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             });
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(STHREADS, 1) small_levels_f32_kernel(F32Args a
             }
             if (!alive) break;
             if (level + 1 < n_levels) {
-                if (!main_grid_barrier(a.meta, (unsigned)level * active_ctas, a.timeout_ns, abort, tid)) alive = false;
+                if (!main_grid_barrier(a.meta, &a.meta[META_BARRIER], (unsigned)level * active_ctas, a.timeout_ns, abort, tid)) alive = false;
             }
             stamp(level, 7, true);
         }

@@ -48,6 +48,7 @@ struct PassSlot {
     int ek_pos[ET_MAX];     // its position in level order (rows of the bf16 copy of h), when positions are known
     int ep[ET_MAX];         // row of the parent inside the tile
     int nodes[NT_MAX];      // node ids of the tile's rows
+    int prow[NT_MAX];       // their rows in the arrays kept by level order: position in level order minus the leaf count
     int eoff[NT_MAX + 1];   // prefix of the rows' child counts
     int pos0, m, ne, et0;   // first position and rows of the tile, its edges, first edge of this pass
 };
@@ -102,11 +103,30 @@ struct DescribeArgs {
     int first_level, n_levels, grp, n_grp, active_grp, nt_max;
     int32_t* meta;       // debug checks: where the first offending index is recorded
     int n_nodes, n_edges, debug;
+    // tree partition (G > 0): the nodes group `grp` has on a level are gperm[goff[level * G + grp] .. goff[level * G + grp + 1])
+    // and the group takes all of their tiles itself; else a level's tiles are dealt out over the active groups
+    const int32_t* gperm;
+    const int32_t* goff;
+    int G, n_leaves;
 };
+
+// Range of the nodes this group has on a level, and which array lists them.
+__device__ __forceinline__ void group_level(const DescribeArgs& d, int level, int& lo, int& hi) {
+    if (d.G > 0) {
+        lo = d.goff[(long long)level * d.G + d.grp];
+        hi = d.goff[(long long)level * d.G + d.grp + 1];
+        if (d.debug && !(dbg_ok(d.meta, CHECK_LEVEL_PTR, lo, (long long)d.n_nodes + 1, level) &&
+                         dbg_ok(d.meta, CHECK_LEVEL_PTR, hi, (long long)d.n_nodes + 1, level) &&
+                         dbg_ok(d.meta, CHECK_LEVEL_PTR, hi - lo, (long long)d.n_nodes + 1, level)))
+            lo = hi = 0;
+    } else {
+        checked_level(d.level_ptr, level, d.n_nodes, d.meta, d.debug, lo, hi);
+    }
+}
 
 // The loop of the description warps (threads MAIN_THREADS .. STHREADS-1 of the CTA; tm = index among them).
 // Walks the same (level, tile, pass) sequence as the arithmetic warps, up to two passes ahead of them.
-// stage_tile(pos0, m, tile_count, tm) is called once per tile after its first slot was acquired and may start
+// stage_tile(slot, m, tile_count, tm) is called once per tile after its first slot was filled in and may start
 // asynchronous copies of per-tile data (they are awaited before the slot is published).
 // Every wait is bounded; a wait that runs out raises *abort, which ends both loops.
 template <class StageTile>
@@ -118,21 +138,30 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
     bool alive = true;
     for (int level = d.first_level; level < d.n_levels && alive; ++level) {
         int lo, hi;
-        checked_level(d.level_ptr, level, d.n_nodes, d.meta, d.debug, lo, hi);
-        const int nt = tile_nodes(hi - lo, d.nt_max, d.n_grp);
+        group_level(d, level, lo, hi);
+        const int nt = tile_nodes(hi - lo, d.nt_max, d.G > 0 ? 1 : d.n_grp);
         const int tiles = (hi - lo + nt - 1) / nt;
-        for (int tile = d.grp; tile < tiles && alive; tile += d.active_grp, ++tcount) {
+        const int32_t* order = d.G > 0 ? d.gperm : d.perm;
+        for (int tile = d.G > 0 ? 0 : d.grp; tile < tiles && alive; tile += d.G > 0 ? 1 : d.active_grp, ++tcount) {
             const int pos0 = lo + tile * nt, m = min(nt, hi - pos0);
             // rows of the tile and the prefix of their child counts
-            int v = -1, eb = 0, incl = 0;
+            int v = -1, eb = 0, incl = 0, prow = 0;
             if (tm < NT_MAX) {
-                if (tm < m) v = d.perm[pos0 + tm];
+                if (tm < m) v = order[pos0 + tm];
                 if (d.debug && tm < m && !dbg_ok(d.meta, CHECK_PERM, v, d.n_nodes, pos0 + tm)) v = -1;  // a row without a node: no edges, nothing stored
                 int cnt = 0;
                 if (v >= 0) { eb = d.child_ptr[v]; cnt = d.child_ptr[v + 1] - eb; }
                 if (d.debug && !(dbg_ok(d.meta, CHECK_EDGE_PTR, eb, (long long)d.n_edges + 1, pos0 + tm) &&
                                  dbg_ok(d.meta, CHECK_EDGE_PTR, cnt, (long long)d.n_edges - eb + 1, pos0 + tm)))
                     eb = cnt = 0;
+                // row of the node in the arrays kept by level order (the input projection's P, the bf16 copy of h)
+                if (v >= 0) {
+                    prow = pos0 + tm - d.n_leaves;
+                    if (d.G > 0) {
+                        prow = d.inv[v] - d.n_leaves;
+                        if (d.debug && !dbg_ok(d.meta, CHECK_POSITION, prow, (long long)d.n_nodes - d.n_leaves, v)) { v = -1; eb = cnt = 0; prow = 0; }
+                    }
+                }
                 incl = cnt;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -152,6 +181,7 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
                 PassSlot& S = R.slot[s];
                 if (tm < NT_MAX) {
                     S.nodes[tm] = v;
+                    S.prow[tm] = prow;
                     S.eoff[tm + 1] = incl;
                     R.t_ebeg[tm] = eb;
                 }
@@ -159,8 +189,8 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
                     S.eoff[0] = 0;
                     S.pos0 = pos0; S.m = m; S.ne = ne; S.et0 = et0;
                 }
-                if (et0 == 0) stage_tile(pos0, m, tcount, tm);
-                named_bar(BAR_META, META_THREADS);  // eoff and t_ebeg of this pass are in place
+                named_bar(BAR_META, META_THREADS);  // nodes, prow, eoff and t_ebeg of this pass are in place
+                if (et0 == 0) stage_tile(S, m, tcount, tm);
                 if (tm < et) {
                     const int e = et0 + tm;
                     int pr = 0, kid = 0, kpos = 0;
@@ -193,16 +223,18 @@ __device__ __forceinline__ void describe_passes(const DescribeArgs& d, Ring& R, 
 // counter meta[META_BARRIER].  Bounded by timeout_ns; on expiry the timeout word is raised (which releases every
 // other waiter) and *abort is set.  Returns with all MAIN_THREADS threads synchronised, and the same verdict in all
 // of them: false when the wait was given up here or *abort was seen raised by anybody.
-__device__ __forceinline__ bool main_grid_barrier(int32_t* meta, unsigned target, unsigned long long timeout_ns,
+// `counter` is meta[META_BARRIER] for a barrier over the whole grid, or the counter of one group of CTAs that walks its
+// own trees (then `target` counts that group's CTAs only).
+__device__ __forceinline__ bool main_grid_barrier(int32_t* meta, int32_t* counter, unsigned target, unsigned long long timeout_ns,
                                                   volatile int* abort, int tid) {
     named_bar(BAR_MAIN, MAIN_THREADS);  // every store of the arithmetic warps is ordered before the release below
     if (tid == 0) {
-        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(&meta[META_BARRIER]) : "memory");
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(counter) : "memory");
         const unsigned long long t0 = global_ns();
         unsigned spins = 0;
         while (true) {
             int seen;
-            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(&meta[META_BARRIER]) : "memory");
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if ((unsigned)seen >= target) break;
             if ((++spins & 15u) == 0) {
                 if (atomicAdd(&meta[META_TIMEOUT], 0) != 0) { *abort = 1; break; }

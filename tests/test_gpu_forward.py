@@ -502,3 +502,28 @@ def test_debug_checks_report_a_schedule_that_does_not_fit_the_forest(precision, 
     torch.cuda.synchronize()
     assert jdb.jdb_debug_report(sched)[0] == 0
     check(w, hh[:, :w.H].cpu().numpy(), cc[:, :w.H].cpu().numpy(), TOL_FP32 if precision == "fp32" else TOL_BF16)
+
+
+def test_tree_partitioned_cooperative_loop_agrees_bit_for_bit_with_grid_barriers():
+    """The cooperative bf16 loop ends every level in a barrier over the whole grid, or (JDB_TUNE_TREE_GROUPS) partitions
+    the forest by tree over its groups of CTAs, which then synchronise inside a group only.  A node's arithmetic does
+    not depend on which tile it shares with whom, so both give the same bits: on a deep forest and on small ragged
+    ones."""
+    w = wl.make_workload(4, n_trees=256)
+    h0, c0, _ = run_forward(w, pad_ld=True)
+    h1, c1, _ = run_forward(w, pad_ld=True, tuning=jdb.TUNE_SET | jdb.TUNE_TREE_GROUPS)
+    h2, c2, _ = run_forward(w, pad_ld=True, tuning=jdb.TUNE_SET | jdb.TUNE_TREE_GROUPS, flags=jdb.FLAG_DEBUG_CHECKS)
+    assert np.array_equal(h0, h1) and np.array_equal(c0, c1) and np.array_equal(h0, h2) and np.array_equal(c0, c2)
+    check(w, h1, c1, TOL_BF16_MATCHED, quantize=matched(w))
+    parents = [[-1, 0, 0, 1, 1, 1, 2, 5, 5, 5, 5], [-1] + [0] * 140, [-1, 0, 1, 2, 3], [-1], [-1] + list(range(60))] * 40
+    for H in (40, 150):
+        w = wl.make_custom(parents, D=72, H=H, seed=800 + H, precision="bf16", bias="random")
+        rng = np.random.default_rng(H)
+        g, new_id = wl.relabel(w.forest, rng)
+        tok = np.empty_like(w.token)
+        tok[new_id] = w.token
+        w.forest, w.token = g, tok
+        h0, c0, _ = run_forward(w, pad_ld=True)
+        h1, c1, _ = run_forward(w, pad_ld=True, tuning=jdb.TUNE_SET | jdb.TUNE_TREE_GROUPS)
+        assert np.array_equal(h0, h1) and np.array_equal(c0, c1)
+        check(w, h1, c1, TOL_BF16_MATCHED, quantize=matched(w))
