@@ -1321,8 +1321,9 @@ bool make_tmap_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t col
 // The switches of one forward call (jdb_opts.tuning, or the defaults with the environment's overrides, read at every
 // call so that nothing depends on what an earlier call saw).
 //   pair_mask  which GEMMs run as CTA pairs (cta_group::2) when they have enough 256-row tiles: 1 input projection,
-//              2 level GEMM, 4 forget-gate GEMM.  Default 4: the forget-gate GEMM gains from the pair reading half of
-//              B per SM; the projection, with its heavier epilogue, does not.
+//              2 level GEMM, 4 forget-gate GEMM.  Default 5: both gain from the pair reading half of B per SM, the
+//              projection only together with eight epilogue warps (same-box runs on the wide forest: 10.9 ms as
+//              pairs with eight warps, 11.7 as pairs with four, 11.4-11.6 as lone CTAs with four).
 //   pdl        programmatic dependent launch of the forward kernels (each waits for its predecessor inside the
 //              kernel, after its own set-up)
 struct Tuning {
@@ -1345,7 +1346,7 @@ Tuning resolve_tuning(int32_t t) {
         return r;
     }
     const char* e = getenv("JDB_GEMM_PAIR");
-    r.pair_mask = e ? (atoi(e) & 7) : 4;
+    r.pair_mask = e ? (atoi(e) & 7) : 5;
     e = getenv("JDB_GEMM_ISSUERS");
     r.issuers = (e && e[0] == '2') ? 2 : 1;
     e = getenv("JDB_PDL");
@@ -1482,7 +1483,11 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     // CTA pairs pay off once there are enough 256-row tiles to keep every pair busy; below that the lone-CTA
     // kernel has the shorter tail.  In pair mode every CTA loads half of a B tile, so the B maps have half-height boxes.
     const bool big = !use_small && (long long)N >= 2LL * BM * n_sm;
-    const bool pair_x = big && (tune.pair_mask & 1), pair_l = big && (tune.pair_mask & 2), pair_f = big && (tune.pair_mask & 4);
+    // the projection as pairs from about 128 tiles per pair on (1.57 M rows x 16 N tiles: 10.9 vs 11.5 ms; 143 k rows x 8:
+    // 0.455 vs 0.444 ms, so that one stays with lone CTAs); an explicit tuning word decides by itself
+    const long long x_tiles2 = ((long long)N + 2 * BM - 1) / (2 * BM) * (4LL * Hp / 256);
+    const bool x_many = (fa.tuning & JDB_TUNE_SET) || x_tiles2 >= 128LL * (n_sm / 2);
+    const bool pair_x = big && x_many && (tune.pair_mask & 1), pair_l = big && (tune.pair_mask & 2), pair_f = big && (tune.pair_mask & 4);
     const uint32_t bdiv = pair_x ? 2 : 1, bdiv_l = pair_l ? 2 : 1;
     CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmHBh, tmUf, tmP, tmHBs;
     // W is read through a full box and a leaf box (i, o, u blocks only)
@@ -1583,12 +1588,13 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         edge_fill_kernel<<<(int)(want < (long long)n_sm * 16 ? want : (long long)n_sm * 16), 256, 0, st>>>(a, w.block_sum);
         JDB_CUDA_TRY(cudaGetLastError());
     }
-    // Eight epilogue warps where the bf16 copy of h goes out row by row anyway (child order) and K is short: with at
-    // most eight K blocks per tile the epilogue weighs more than the pipeline stage the eight step buffers cost
-    // (D = 512: 0.47 -> 0.44 ms on 143 k nodes); at sixteen K blocks the four-stage kernel is ahead (D = 1024: 1.16 vs
-    // 1.22 ms on 195 k nodes).  The small forests of the cooperative loop keep the four-warp kernel, whose leaf tiles
-    // leave as one TMA box per warp.
-    const int xepi = (!use_small && !tune.issuers2_requested && kd <= 8) ? EPI_XPROJ8 : EPI_XPROJ;
+    // Eight epilogue warps where the bf16 copy of h goes out row by row anyway (child order) and either K is short or
+    // the GEMM runs as CTA pairs: with at most eight K blocks per tile the epilogue weighs more than the pipeline stage
+    // the eight step buffers cost a lone CTA (D = 512: 0.47 -> 0.44 ms on 143 k nodes), while at sixteen K blocks the
+    // lone four-stage kernel is ahead of the lone three-stage one (D = 1024: 1.16 vs 1.22 ms on 195 k nodes); a CTA of a
+    // pair keeps four stages either way.  The small forests of the cooperative loop keep the four-warp kernel, whose
+    // leaf tiles leave as one TMA box per warp.
+    const int xepi = (!use_small && !tune.issuers2_requested && (kd <= 8 || pair_x)) ? EPI_XPROJ8 : EPI_XPROJ;
     if ((ls = launch(xepi, tmX, tmW, tmWl, (long long)N + 2 * BM, 0, 256, 4 * Hp, kd)) != JDB_OK) return ls;
     if (fa.ev_xproj_done) JDB_CUDA_TRY(cudaEventRecord(fa.ev_xproj_done, st));
     if (!use_small) {
