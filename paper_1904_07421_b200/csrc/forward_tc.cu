@@ -47,6 +47,10 @@ constexpr int GEMM1_THREADS = 224;  // warp 0: TMA producer, warps 1 and 6: MMA 
 // warps, two per TMEM lane quarter and per scheduler, which take the steps of a tile alternately.
 constexpr int GEMMF_THREADS = 320;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
 __host__ __device__ constexpr int gemm_threads(int epi) { return (epi == 2 || epi == 3) ? GEMMF_THREADS : GEMM1_THREADS; }
+// the CTA-pair forget-gate GEMM runs sixteen epilogue warps (four per scheduler): warp 0 producer, 1 issuer, 2-17 epilogue
+constexpr int GEMMF2_THREADS = 576;
+__host__ __device__ constexpr int gemm2_threads(int epi) { return epi == 2 ? GEMMF2_THREADS : gemm_threads(epi); }
+__host__ __device__ constexpr int epi_warps2(int epi) { return epi == 2 ? 16 : (epi == 3 ? 8 : 4); }
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;
 constexpr int TMEM_COLS = 512;  // two accumulator buffers of up to 256 columns
 
@@ -134,11 +138,15 @@ constexpr int GEMM_SMEM_STORE = GEMM_SMEM + 4 * EPI_STEP_FLOATS * 4;   // input 
 constexpr int F_STEP_FLOATS = 2 * 32 * 16;
 constexpr int F_STAGES = 3;
 constexpr int F_WARPS = 8;
-// step buffers per warp: the copies of a step start F_RING - 1 steps ahead.  A CTA of a pair holds half of B per
-// stage, which leaves room for one more buffer per warp than a lone CTA has.
-__host__ __device__ constexpr int f_ring(bool pair) { return pair ? 3 : 2; }
-constexpr int F_SCRATCH_BYTES = F_WARPS * f_ring(false) * F_STEP_FLOATS * 4;
-constexpr int F_SCRATCH2_BYTES = F_WARPS * f_ring(true) * F_STEP_FLOATS * 4;
+// A lone CTA: eight epilogue warps, each walking 128 of the tile's 256 edges.  A CTA of a pair holds half of B per
+// stage, which leaves room for sixteen warps (64 edges each) with three pipeline stages.  Two step buffers per warp: the
+// copies of a step start one step ahead (a third buffer, tried in the pair kernel, changed nothing).
+__host__ __device__ constexpr int f_warps(bool pair) { return pair ? 16 : 8; }
+__host__ __device__ constexpr int f_seg(bool pair) { return pair ? 64 : 128; }
+__host__ __device__ constexpr int f_ring(bool pair) { return 2; }
+constexpr int F_SCRATCH_BYTES = f_warps(false) * f_ring(false) * F_STEP_FLOATS * 4;
+constexpr int F_SCRATCH2_BYTES = f_warps(true) * f_ring(true) * F_STEP_FLOATS * 4;
+constexpr int STAGES2_F = 3;
 constexpr int GEMM_SMEM_F = F_STAGES * STAGE_BYTES + F_SCRATCH_BYTES + 1024;
 constexpr int X8_STAGES = 3;
 constexpr int GEMM_SMEM_X8 = X8_STAGES * STAGE_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;   // eight warps, one step buffer each
@@ -379,7 +387,6 @@ __device__ __forceinline__ void xproj_internal_tile_tma(const TcArgs& a, const T
 // the child's c: [16 edges][32 floats] arrays in shared memory, filled by 16-byte asynchronous copies one step ahead
 // (eight lanes per edge row) and read one float per lane, free of bank conflicts.
 constexpr int F_EDGES = 256;      // edges per tile (the MMA's N)
-constexpr int F_SEG = 128;        // edges per epilogue warp
 // pr, kd: parent row and child node id of this lane's edges lane + 32 i of the segment, chosen for the step by the caller
 __device__ __forceinline__ void forget_fetch(const TcArgs& a, int j_base, int lane, int st, int pr_sel, int kd_sel, uint32_t buf,
                                              float* bufp) {
@@ -420,13 +427,16 @@ struct Segment {
 __device__ __forceinline__ int sel4(const int (&v)[4], int i) { return i == 0 ? v[0] : i == 1 ? v[1] : i == 2 ? v[2] : v[3]; }
 __device__ __forceinline__ unsigned sel4u(const unsigned (&v)[4], int i) { return i == 0 ? v[0] : i == 1 ? v[1] : i == 2 ? v[2] : v[3]; }
 
+template <int SEG>
 __device__ __forceinline__ Segment segment_of(const TcArgs& a, int slot0, int row_end, int lane) {
+    constexpr int NI = SEG / 32;
     Segment sg;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int sl = slot0 + 32 * i + lane;
         sg.pr[i] = sg.kd[i] = -1;
-        if (sl < row_end) {
+        sg.heads[i] = 0;
+        if (i < NI && sl < row_end) {
             sg.pr[i] = a.slot_par[sl];
             sg.kd[i] = a.slot_child[sl];
             if (a.debug && (!dbg_ok(a.meta, CHECK_PARENT_ROW, sg.pr[i], a.n_int_bound, sl) ||
@@ -435,19 +445,19 @@ __device__ __forceinline__ Segment segment_of(const TcArgs& a, int slot0, int ro
         }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < NI; ++i) {
         int prev = __shfl_up_sync(0xffffffffu, sg.pr[i], 1);
         const int carry = __shfl_sync(0xffffffffu, sg.pr[i > 0 ? i - 1 : 0], 31);
         if (lane == 0) prev = carry;
         sg.heads[i] = __ballot_sync(0xffffffffu, (i == 0 && lane == 0) || sg.pr[i] != prev);
     }
-    const int n_valid = min(max(row_end - slot0, 0), F_SEG);
+    const int n_valid = min(max(row_end - slot0, 0), SEG);
     const int p_first = __shfl_sync(0xffffffffu, sg.pr[0], 0);
     sg.cont_before = p_first >= 0 && a.eoff[p_first] != slot0;
     sg.cont_after = false;
-    if (n_valid == F_SEG) {
-        const int p_last = __shfl_sync(0xffffffffu, sg.pr[3], 31);
-        sg.cont_after = p_last >= 0 && a.eoff[p_last + 1] != slot0 + F_SEG;
+    if (n_valid == SEG) {
+        const int p_last = __shfl_sync(0xffffffffu, sg.pr[NI - 1], 31);
+        sg.cont_after = p_last >= 0 && a.eoff[p_last + 1] != slot0 + SEG;
     }
     return sg;
 }
@@ -581,8 +591,8 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
         }
         cp_async_wait<0>();
     } else if (EPI == EPI_F) {
-        // eight warps: lane quarter = 32 hidden units, segment = the first or the second 128 edges of the tile
-        constexpr int RING = f_ring(PAIR), STEPS = F_SEG / 16;
+        // eight or sixteen warps: lane quarter = 32 hidden units, segment = 128 or 64 consecutive edges of the tile
+        constexpr int RING = f_ring(PAIR), F_SEG = f_seg(PAIR), STEPS = F_SEG / 16;
         const int seg = (warp - 2) >> 2;
         float* ring = scratch + (warp - 2) * (RING * F_STEP_FLOATS);
         const uint32_t ring_addr = smem_u32(ring);
@@ -592,7 +602,7 @@ __device__ __forceinline__ void epilogue_warps(const TcArgs& a, const CUtensorMa
             const int j_base = ti.n_tile * TMH + rank * BM + quarter * 32, j = j_base + lane;
             const bool j_ok = j < a.Hp;
             const int slot0 = ti.row0 + seg * F_SEG;
-            const Segment sg = segment_of(a, slot0, ti.row_end, lane);
+            const Segment sg = segment_of<F_SEG>(a, slot0, ti.row_end, lane);
             // the first steps' copies start before the accumulator is ready: they land while the tile's products run
 #pragma unroll
             for (int st = 0; st < RING - 1; ++st) {
@@ -864,17 +874,18 @@ constexpr int STAGES2 = 6, STAGES2_LEVEL = 4;
 constexpr int STAGE2_BYTES = A_BYTES + B_BYTES_MAX / 2;
 constexpr int GEMM2_SMEM = STAGES2 * STAGE2_BYTES + 4 * EPI_STEP_FLOATS * 4 + 1024;
 constexpr int GEMM2_SMEM_LEVEL = STAGES2_LEVEL * STAGE2_BYTES + EPI_SCRATCH_BYTES + 1024;
-constexpr int GEMM2_SMEM_F = STAGES2_LEVEL * STAGE2_BYTES + F_SCRATCH2_BYTES + 1024;
+constexpr int GEMM2_SMEM_F = STAGES2_F * STAGE2_BYTES + F_SCRATCH2_BYTES + 1024;
 static_assert(GEMM2_SMEM_F <= 227 * 1024 - 256, "pair forget GEMM shared memory");
 constexpr int GEMM2_SMEM_X8 = STAGES2_LEVEL * STAGE2_BYTES + 8 * EPI_STEP_FLOATS * 4 + 1024;
 static_assert(GEMM2_SMEM_LEVEL <= 227 * 1024 - 256, "pair level GEMM shared memory");
 
 template <int EPI>
-__global__ void __launch_bounds__(gemm_threads(EPI), 1)
+__global__ void __launch_bounds__(gemm2_threads(EPI), 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmB_leaf, const __grid_constant__ CUtensorMap tmP,
                const __grid_constant__ CUtensorMap tmHBs, TcArgs a, int level, int bn, int n_total, int kblocks) {
-    constexpr int NST2 = EPI == EPI_XPROJ ? STAGES2 : STAGES2_LEVEL;   // the kernels with rings or eight step buffers give up two stages
+    // the kernels with rings or eight step buffers give up two stages, the sixteen-warp forget-gate kernel three
+    constexpr int NST2 = EPI == EPI_XPROJ ? STAGES2 : EPI == EPI_F ? STAGES2_F : STAGES2_LEVEL;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_full[NST2], bar_empty[NST2], bar_tfull[2], bar_tempty[2];
     __shared__ uint32_t s_tmem_base;
@@ -912,7 +923,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_tfull[b]), 1);
-            mbar_init(smem_u32(&bar_tempty[b]), 64 * epi_warps(EPI));  // the epilogue threads of both CTAs
+            mbar_init(smem_u32(&bar_tempty[b]), 64 * epi_warps2(EPI));  // the epilogue threads of both CTAs
         }
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -1007,7 +1018,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             if (!ok && lane == 0) *abort = 1;
         }
-    } else if (warp >= 2 && warp <= 1 + epi_warps(EPI)) {
+    } else if (warp >= 2 && warp <= 1 + epi_warps2(EPI)) {
         epilogue_warps<EPI, true>(a, &tmP, &tmHBs, reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + NST2 * STAGE2_BYTES),
                                   tmem_base, bar_tfull, bar_tempty, abort, warp, lane, pair, n_pairs, total_tiles, n_tiles, lo, hi,
                                   bn, n_leaves, mt_leaf, (int)rank);
@@ -1547,7 +1558,7 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         int pairs = (int)(tiles2 < n_sm / 2 ? (tiles2 > 0 ? tiles2 : 1) : n_sm / 2);
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(2 * pairs);
-        cfg.blockDim = dim3(gemm_threads(epi));
+        cfg.blockDim = dim3(gemm2_threads(epi));
         cfg.dynamicSmemBytes = epi == EPI_LEVEL ? GEMM2_SMEM_LEVEL : epi == EPI_F ? GEMM2_SMEM_F : epi == EPI_XPROJ8 ? GEMM2_SMEM_X8 : GEMM2_SMEM;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];

@@ -223,18 +223,25 @@ def test_config5_sampled():
 
 
 def _variants_agree_bit_for_bit(index, tunings, n_trees=None):
-    """The GEMM switches change how a product is scheduled (CTA pairs, issuer warps, launch overlap, store path), never
-    its arithmetic: every row of h and c must come out with the same bits."""
+    """The GEMM switches change how a product is scheduled (CTA pairs, issuer warps, launch overlap, store path, how x
+    is fetched), never its arithmetic: every row of h and c must come out with the same bits.  One exception by
+    design: the forget-gate GEMM adds a parent's f c_k in runs of 128 edge slots as lone CTAs and of 64 as CTA pairs, so
+    the two groups of variants agree with each other to fp32 rounding order only, which a bf16 rounding of h further up
+    the tree can turn into one bf16 unit in the last place of an operand: they are held to 2e-3."""
     w = wl.make_workload(index, n_trees=n_trees)
-    ref = None
+    ref = {}
     for t in tunings:
         h, c, _ = run_forward(w, bench_ld=True, tuning=t, to_host=False)
-        if ref is None:
-            ref = (h, c, t)
+        pair_forget = t == 0 or bool(t & jdb.TUNE_PAIR_FORGET)
+        if pair_forget not in ref:
+            ref[pair_forget] = (h, c, t)
             continue
-        assert torch.equal(h, ref[0]) and torch.equal(c, ref[1]), (t, ref[2])
+        assert torch.equal(h, ref[pair_forget][0]) and torch.equal(c, ref[pair_forget][1]), (t, ref[pair_forget][2])
         del h, c
-    return w, ref[0], ref[1]
+    if len(ref) == 2:
+        assert float((ref[True][0] - ref[False][0]).abs().max()) <= 2e-3 and float((ref[True][1] - ref[False][1]).abs().max()) <= 2e-3
+    h, c, _ = ref[True] if True in ref else ref[False]
+    return w, h, c
 
 
 _TUNINGS = [jdb.TUNE_SET,                                                          # lone CTAs everywhere
