@@ -249,12 +249,12 @@ MEASURED_TRAFFIC = {
     ("small_levels_kernel", 4): 896706560,              # whole workload captured, one launch
     # per-level loop = all childsum_kernel, gemm_tc_kernel<EPI_F> and gemm_tc_kernel<EPI_LEVEL> launches of one step
     ("per-level loop", 3): 1656050000,                  # whole workload captured (12 levels, 36 launches)
-    # captured on 8192 of the 65536 trees (194583 nodes: 2765 MB) and scaled by the node count: every row is read and
+    # captured on 8192 of the 65536 trees (194583 nodes: 2775 MB) and scaled by the node count: every row is read and
     # written a fixed number of times, so traffic grows in proportion
-    ("per-level loop", 5): int(2765.0e6 * (1571637 / 194583)),
-    # input projection of workload 5 (four-warp kernel, rows of the bf16 copy to their slots): one launch captured on the
-    # same 8192 trees (408.59 MB read, 2034.67 MB written), scaled
-    ("gemm_tc_kernel<EPI_XPROJ>", 5): int(2443266816 * (1571637 / 194583)),
+    ("per-level loop", 5): int(2775.2e6 * (1571637 / 194583)),
+    # input projection of workload 5 (CTA pairs, eight epilogue warps): one launch captured on the same 8192 trees
+    # (409.06 MB read, 2035.62 MB written), scaled
+    ("gemm_tc2_kernel<EPI_XPROJ8>", 5): int(2444.68e6 * (1571637 / 194583)),
 }
 
 
@@ -291,7 +291,7 @@ def roofline_of(job, phases, t_step_s, pk):
     else:
         lkernel = "per-level loop"
     phases_out = {
-        "input_projection": {"kernel": "gemm_tc_kernel<EPI_XPROJ>" if w.precision == "bf16" else "xproj_simt_kernel",
+        "input_projection": {"kernel": "tcgen05 GEMM (gemm_tc_kernel / gemm_tc2_kernel)" if w.precision == "bf16" else "xproj_simt_kernel",
                              "ms": xproj_ms, "flops": xflops, "tflops": x_ach,
                              "frac_of_tensor_peak": x_ach / tensor_peak if w.precision == "bf16" else None},
         "level_loop": {"kernel": lkernel, "ms": lvl_ms, "algorithmic_bytes": lbytes, "design_bytes": ldesign,
@@ -300,7 +300,10 @@ def roofline_of(job, phases, t_step_s, pk):
         "schedule_ms": statistics.mean(p[2] for p in phases),
     }
     if w.precision == "bf16" and xproj_ms >= lvl_ms:
-        kernel = "gemm_tc_kernel<EPI_XPROJ>"
+        # the library's own choice: CTA pairs with eight epilogue warps from 128 tiles per pair on (148 SMs)
+        Hp = (H + 63) // 64 * 64
+        many = not job.small and ((N + 255) // 256) * (4 * Hp // 256) >= 128 * 74
+        kernel = "gemm_tc2_kernel<EPI_XPROJ8>" if many else "gemm_tc_kernel<EPI_XPROJ>"
         roof = {"bound": "tensor", "kernel": kernel, "achieved": x_ach, "peak": tensor_peak, "unit": "TFLOP/s",
                 "frac": x_ach / tensor_peak, "frac_of_sustained_peak": x_ach / pk["bf16_tflops_sustained"]}
     else:
