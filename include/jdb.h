@@ -61,7 +61,7 @@ enum {
 enum {
     JDB_TUNE_SET = 1,
     JDB_TUNE_PAIR_XPROJ = 2,    /* input-projection GEMM as CTA pairs (forests of at least 256 rows per SM); default   */
-    JDB_TUNE_PAIR_LEVEL = 4,    /* per-level gate GEMM as CTA pairs                                                  */
+    JDB_TUNE_PAIR_LEVEL = 4,    /* per-level gate GEMM as CTA pairs (launches with at least 32 tiles per pair); default */
     JDB_TUNE_PAIR_FORGET = 8,   /* per-level forget-gate GEMM as CTA pairs (launches with at least 32 tiles per pair); default */
     JDB_TUNE_TWO_ISSUERS = 16,  /* two MMA-issuing warps per lone CTA, half of the tile's columns each               */
     JDB_TUNE_NO_PDL = 32,       /* ordinary launches instead of programmatic dependent launches                      */

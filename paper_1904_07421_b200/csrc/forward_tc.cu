@@ -1332,7 +1332,8 @@ bool make_tmap_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t col
 // The switches of one forward call (jdb_opts.tuning, or the defaults with the environment's overrides, read at every
 // call so that nothing depends on what an earlier call saw).
 //   pair_mask  which GEMMs run as CTA pairs (cta_group::2) when they have enough 256-row tiles: 1 input projection,
-//              2 level GEMM, 4 forget-gate GEMM.  Default 5: both gain from the pair reading half of B per SM, the
+//              2 level GEMM, 4 forget-gate GEMM.  Default 7 (the per-level GEMMs launch by launch, from 32 tiles per
+//              pair on; the gate GEMM gains about 2 % on the wide forest): all gain from the pair reading half of B per SM, the
 //              projection only together with eight epilogue warps (same-box runs on the wide forest: 10.9 ms as
 //              pairs with eight warps, 11.7 as pairs with four, 11.4-11.6 as lone CTAs with four).
 //   pdl        programmatic dependent launch of the forward kernels (each waits for its predecessor inside the
@@ -1357,7 +1358,7 @@ Tuning resolve_tuning(int32_t t) {
         return r;
     }
     const char* e = getenv("JDB_GEMM_PAIR");
-    r.pair_mask = e ? (atoi(e) & 7) : 5;
+    r.pair_mask = e ? (atoi(e) & 7) : 7;
     e = getenv("JDB_GEMM_ISSUERS");
     r.issuers = (e && e[0] == '2') ? 2 : 1;
     e = getenv("JDB_PDL");
@@ -1499,16 +1500,17 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
     const long long x_tiles2 = ((long long)N + 2 * BM - 1) / (2 * BM) * (4LL * Hp / 256);
     const bool x_many = (fa.tuning & JDB_TUNE_SET) || x_tiles2 >= 128LL * (n_sm / 2);
     const bool pair_x = big && x_many && (tune.pair_mask & 1), pair_l = big && (tune.pair_mask & 2), pair_f = big && (tune.pair_mask & 4);
-    const uint32_t bdiv = pair_x ? 2 : 1, bdiv_l = pair_l ? 2 : 1;
-    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmHB, tmHBh, tmUf, tmP, tmHBs;
+    const uint32_t bdiv = pair_x ? 2 : 1;
+    CUtensorMap tmX, tmW, tmWl, tmHS, tmUiou, tmUiouh, tmHB, tmHBh, tmUf, tmP, tmHBs;
     // W is read through a full box and a leaf box (i, o, u blocks only)
     bool ok = (a.x_gather ? make_tmap(&tmX, fa.x, n, (uint64_t)D, (uint64_t)fa.ldx, 1)    // one-row boxes for the gathers
                           : make_tmap(&tmX, w.xb, n, (uint64_t)D, (uint64_t)Dp, BM)) &&
               make_tmap(&tmW, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 256 / bdiv) &&
               make_tmap(&tmWl, pk + L.off_W, (uint64_t)4 * Hp, (uint64_t)L.Kd, (uint64_t)L.Kd, 192 / bdiv);
-    if (ok && !use_small)   // the per-level launches read their operands through five more maps
+    if (ok && !use_small)   // the per-level launches read their operands through six more maps
         ok = make_tmap(&tmHS, w.hs, ni, (uint64_t)Hp, (uint64_t)Hp, BM) &&
-             make_tmap(&tmUiou, pk + L.off_Uiou, (uint64_t)3 * Hp, (uint64_t)Hp, (uint64_t)Hp, 192 / bdiv_l) &&
+             make_tmap(&tmUiou, pk + L.off_Uiou, (uint64_t)3 * Hp, (uint64_t)Hp, (uint64_t)Hp, 192) &&
+             make_tmap(&tmUiouh, pk + L.off_Uiou, (uint64_t)3 * Hp, (uint64_t)Hp, (uint64_t)Hp, 96) &&   // half per CTA of a pair
              make_tmap(&tmHB, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, F_EDGES) &&        // forget-gate GEMM: B, a tile's 256 edge rows
              make_tmap(&tmHBh, w.hb, n, (uint64_t)Hp, (uint64_t)Hp, F_EDGES / 2) &&   // ... half of them per CTA of a pair
              make_tmap(&tmUf, pk + L.off_Uf, (uint64_t)Hp, (uint64_t)Hp, (uint64_t)Hp, BM);   // ... A, 128 hidden units
@@ -1544,8 +1546,8 @@ jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int 
         const int n_tiles2 = epi == EPI_F ? (Hp + 2 * BM - 1) / (2 * BM) : n_tiles;
         // the forget-gate GEMM decides launch by launch: pairs pay off from about 32 tiles per pair on
         const long long tiles2 = (rows_bound + 2 * BM - 1) / (2 * BM) * n_tiles2;
-        const bool pair = is_xproj(epi) ? pair_x : epi == EPI_LEVEL ? pair_l : (pair_f && tiles2 >= 32LL * (n_sm / 2));
-        const CUtensorMap& tB = (epi == EPI_F && pair) ? tmHBh : tB_full;
+        const bool pair = is_xproj(epi) ? pair_x : ((epi == EPI_LEVEL ? pair_l : pair_f) && tiles2 >= 32LL * (n_sm / 2));
+        const CUtensorMap& tB = (epi == EPI_F && pair) ? tmHBh : (epi == EPI_LEVEL && pair) ? tmUiouh : tB_full;
         if (!pair) {
             const long long lone_tiles = epi == EPI_F ? (rows_bound + F_EDGES - 1) / F_EDGES * n_tiles : 0;
             const int grid = epi == EPI_F ? (int)(lone_tiles < n_sm ? (lone_tiles > 0 ? lone_tiles : 1) : n_sm) : gemm_grid(rows_bound, n_tiles);
