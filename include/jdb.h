@@ -243,6 +243,34 @@ jdb_status jdb_relatedness_head(const float *h, int64_t ldh, int32_t n_nodes, co
                                 const float *bq, int32_t H, int32_t Hs, int32_t K, float *y, float *p, int32_t *bad_flag,
                                 void *stream);
 
+/* ---- backward pass (training: the listing of Section 4.3 calls backward() inside the batching scope) ---------- */
+
+/* Bytes of device scratch for one backward call.  n_internal_bound as for the forward workspace. */
+size_t jdb_treelstm_backward_workspace_bytes(int32_t n_nodes, int32_t n_edges, int32_t n_internal_bound, int32_t H);
+
+/* Gradients of L = sum_v <grad_h[v], h_v> + <grad_c[v], c_v> for the cell of jdb_treelstm_forward, over the same depth
+ * table with the levels in DESCENDING order (a node's gradient is complete once its parent's level is done; Section 5
+ * reports the training speed-up this pass takes part in).  fp32 throughout.
+ * sched    from jdb_schedule on `forest` (the level count and level offsets are needed on the host: the call copies the
+ *          level table back and synchronises `stream` ONCE before its launches; a schedule from jdb_schedule_async,
+ *          whose counts were never read back, gives JDB_ERR_INVALID_ARG, and so does one whose node, leaf or edge
+ *          totals do not fit this forest).
+ * x        [n_nodes, D] fp32, leading dimension ldx.  W [4H, D], U [4H, H], b [4H]: the natural matrices, fp32
+ *          row-major, gate row blocks (i, o, u, f), as given to jdb_pack_weights.
+ * h, c     [n_nodes, H] fp32, leading dimension ldh: the outputs of the forward pass on the same inputs.
+ * grad_h   [n_nodes, H] fp32, leading dimension ldg: dL/dh of every node (rows of nodes the loss does not see are
+ *          zero); grad_c the same for c, or NULL for zeros.
+ * dW [4H, D], dU [4H, H], db [4H]: outputs, dense, OVERWRITTEN (not accumulated).  dx [n_nodes, D] with leading
+ * dimension lddx, or NULL to skip it.  The sums over nodes and edges behind dW, dU and db are split over CTAs whose
+ * partial sums are added atomically: their last bits can differ from run to run.
+ * ws       device scratch of jdb_treelstm_backward_workspace_bytes bytes, 256-byte aligned.
+ * Everything after the one synchronisation is asynchronous on `stream`; allocates nothing on the device. */
+jdb_status jdb_treelstm_backward(const jdb_forest *forest, const jdb_sched *sched, const float *x, int64_t ldx,
+                                 const float *W, const float *U, const float *b, int32_t D, int32_t H, const float *h,
+                                 const float *c, int64_t ldh, const float *grad_h, const float *grad_c, int64_t ldg,
+                                 float *dW, float *dU, float *db, float *dx, int64_t lddx, void *ws, size_t ws_bytes,
+                                 void *stream);
+
 /* ---- one call from host buffers (what a user without device arrays calls) -------------------- */
 
 /* Device scratch needed by jdb_treelstm_forward_host (CSR, x, schedule, h, c and both workspaces). */

@@ -29,6 +29,7 @@ EXPORTS = [
     "jdb_schedule_async", "jdb_schedule_static", "jdb_packed_weights_bytes", "jdb_pack_weights", "jdb_forward_workspace_bytes",
     "jdb_treelstm_forward", "jdb_sched_status", "jdb_debug_report", "jdb_forward_host_workspace_bytes",
     "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts", "jdb_relatedness_head",
+    "jdb_treelstm_backward_workspace_bytes", "jdb_treelstm_backward",
 ]
 
 
@@ -101,6 +102,11 @@ def lib():
     L.jdb_launch_counts_workspace_bytes.argtypes = [i32]
     L.jdb_launch_counts.restype = C.c_int
     L.jdb_launch_counts.argtypes = [C.POINTER(CForest), C.POINTER(CSched), C.POINTER(CLaunchStats), vp, sz, vp]
+    L.jdb_treelstm_backward_workspace_bytes.restype = C.c_size_t
+    L.jdb_treelstm_backward_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.jdb_treelstm_backward.restype = C.c_int
+    L.jdb_treelstm_backward.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, i64,
+                                        vp, C.c_size_t, vp]
     L.jdb_relatedness_head.restype = C.c_int
     L.jdb_relatedness_head.argtypes = [vp, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
@@ -294,6 +300,39 @@ def jdb_relatedness_head(h: torch.Tensor, left: torch.Tensor, right: torch.Tenso
     if st != OK:
         raise JdbError(st, "jdb_relatedness_head")
     return y[:P], (p[:P] if want_p else None), bad
+
+
+def jdb_treelstm_backward(forest: Forest, sched: Schedule, x: torch.Tensor, W: torch.Tensor, U: torch.Tensor, b: torch.Tensor,
+                          h: torch.Tensor, c: torch.Tensor, grad_h: torch.Tensor, grad_c: Optional[torch.Tensor] = None,
+                          want_dx: bool = True, ws: Optional[torch.Tensor] = None, stream=None):
+    """(dW [4H, D], dU [4H, H], db [4H], dx [n, D] or None) of L = <grad_h, h> + <grad_c, c>; fp32 device tensors.
+
+    h and c are the forward outputs (row stride h.stride(0)); grad_h / grad_c are [n, >= H] with a common row stride.
+    """
+    H4, D = W.shape
+    H = H4 // 4
+    n = forest.n_nodes
+    dev = x.device
+    if x.dtype != torch.float32 or h.dtype != torch.float32 or c.dtype != torch.float32 or grad_h.dtype != torch.float32:
+        raise ValueError("jdb_treelstm_backward computes in fp32: x, h, c and grad_h must be float32")
+    if c.stride(0) != h.stride(0) or (grad_c is not None and grad_c.stride(0) != grad_h.stride(0)):
+        raise ValueError("h and c (and grad_h and grad_c) must share a row stride")
+    W, U, b = (t.to(torch.float32).contiguous() for t in (W, U, b))
+    n_int = n - sched.n_leaves if sched.n_leaves >= 0 else n
+    if ws is None:
+        ws = _device_bytes(lib().jdb_treelstm_backward_workspace_bytes(n, forest.n_edges, n_int, H), dev)
+    dW = torch.empty((4 * H, D), dtype=torch.float32, device=dev)
+    dU = torch.empty((4 * H, H), dtype=torch.float32, device=dev)
+    db = torch.empty(4 * H, dtype=torch.float32, device=dev)
+    dx = torch.empty((max(n, 1), D), dtype=torch.float32, device=dev) if want_dx else None
+    cf, cs = forest.c(), sched.c()
+    st = lib().jdb_treelstm_backward(C.byref(cf), C.byref(cs), _ptr(x), x.stride(0) if n > 0 else D, _ptr(W), _ptr(U), _ptr(b), D, H,
+                                     _ptr(h), _ptr(c), h.stride(0) if n > 0 else H, _ptr(grad_h), _ptr(grad_c),
+                                     grad_h.stride(0) if n > 0 else H, _ptr(dW), _ptr(dU), _ptr(db), _ptr(dx), D, _ptr(ws), ws.numel(),
+                                     _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_treelstm_backward")
+    return dW, dU, db, (dx[:n] if want_dx else None)
 
 
 def jdb_debug_report(sched: Schedule, stream=None):
