@@ -29,6 +29,8 @@ from paper_1904_07421_b200 import workloads as wl  # noqa: E402
 METRIC = "treelstm_forward_nodes_per_sec"
 UNIT = "nodes/s"
 L2_FLUSH_BYTES = 256 << 20
+# fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flops x 1.965 GHz (the part's maximum SM clock)
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
 def peaks():
@@ -461,6 +463,54 @@ def time_head(w: wl.Workload, job: GpuJob, flush, pk, Hs: int = 50, K: int = 5, 
             "frac_of_hbm_peak": bytes_ / (t * 1e-3) / 1e9 / pk["hbm_gbs"], "head_hidden": Hs, "classes": K}
 
 
+def time_training(idx: int, w: wl.Workload, device, flush, steps: int = 5, warmup: int = 3):
+    """One training pass in fp32 (Section 5 reports training beside inference): batching analysis, forward, and the
+    backward pass over the same depth table with the loss on the root states.  Not part of `value`."""
+    import torch
+    from paper_1904_07421_b200 import jdb
+    f = w.forest
+    D, H = w.D, w.H
+    forest = jdb.forest_to_device(f.child_ptr, f.child_idx, device)
+    x = torch.from_numpy(w.x_full()).to(device)
+    W, U, b = (torch.from_numpy(a).to(device) for a in (w.W, w.U, w.b))
+    packed = jdb.jdb_pack_weights(W, U, b, jdb.FP32)
+    sched = jdb.alloc_schedule(f.n_nodes, device)
+    sws = jdb.schedule_workspace(forest)
+    jdb.jdb_schedule(forest, sched, sws)
+    n_int = f.n_nodes - sched.n_leaves
+    fws = jdb.forward_workspace(forest, sched, D, H, jdb.FP32)
+    bws = torch.empty(jdb.lib().jdb_treelstm_backward_workspace_bytes(f.n_nodes, f.n_edges, n_int, H), dtype=torch.uint8, device=device)
+    h = torch.empty((f.n_nodes, H), dtype=torch.float32, device=device)
+    c = torch.empty_like(h)
+    gh = torch.zeros_like(h)
+    rng = np.random.default_rng(11)
+    roots = torch.from_numpy(f.roots.astype(np.int64)).to(device)
+    gh[roots] = torch.from_numpy(rng.standard_normal((f.n_trees, H)).astype(np.float32)).to(device)
+    fwd, bwd = [], []
+    for it in range(warmup + steps):
+        flush.add_(1)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        jdb.jdb_schedule(forest, sched, sws)
+        jdb.jdb_treelstm_forward(forest, sched, x, packed, D, H, jdb.FP32, h=h, c=c, ws=fws)
+        e[1].record()
+        jdb.jdb_treelstm_backward(forest, sched, x, W, U, b, h, c, gh, None, ws=bws)
+        e[2].record()
+        e[2].synchronize()
+        if it >= warmup:
+            fwd.append(e[0].elapsed_time(e[1]))
+            bwd.append(e[1].elapsed_time(e[2]))
+    tf, tb = statistics.median(fwd), statistics.median(bwd)
+    flops_b = 3.0 * (8.0 * f.n_nodes * D * H + 6.0 * n_int * H * H + 2.0 * f.n_edges * H * H)
+    return {"config": idx, "workload": w.name, "nodes": f.n_nodes, "trees": f.n_trees, "D": D, "H": H, "dtype": "f32",
+            "step": "jdb_schedule + jdb_treelstm_forward + jdb_treelstm_backward (loss on the roots)",
+            "forward_ms": tf, "backward_ms": tb, "nodes_per_s": f.n_nodes / ((tf + tb) * 1e-3),
+            "trees_per_s": f.n_trees / ((tf + tb) * 1e-3), "backward_flops": flops_b,
+            "backward_tflops": flops_b / (tb * 1e-3) / 1e12,
+            "backward_frac_of_fp32_alu_peak": flops_b / (tb * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
+            "launches_backward": 4 + 2 + 3 + 3 * max(sched.n_levels - 1, 0) + 1 + 5}
+
+
 def rank_workload(config: int, rank: int, n_trees=None) -> wl.Workload:
     """Every rank draws its own forest of the workload's shape (weak scaling over independent trees)."""
     return wl.make_workload(config, n_trees=n_trees, seed=None if rank == 0 else wl.BASE_SEED + config + 1000 * rank)
@@ -571,6 +621,11 @@ def run_gpu(args):
                 per_config.append(config_entry(idx, wi, ji, ti, args.steps, wi.forest.n_nodes * args.steps / (sum(ti) / 1e3), ri, pf, po))
                 del ji, wi
                 torch.cuda.empty_cache()
+        training = []
+        if args.all_configs and world == 1:
+            for idx in (1, 2, 3, 4):
+                training.append(time_training(idx, wl.make_workload(idx), device, flush))
+                torch.cuda.empty_cache()
         cpu_v, cpu_sample, cpu_trees = time_oracle(w, args.cpu_budget)
         cpu_par = None
         if args.cpu_budget >= 1.0:
@@ -594,6 +649,7 @@ def run_gpu(args):
             "path_frac_of_roofline": path_frac,
             "phases": phases_out,
             "relatedness_head": head,
+            "training": training,
             "batching_ratio": f.n_nodes / max(n_levels_main, 1),   # cells evaluated per batched step: Section 3's batching ratio at cell granularity
             "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample,
                              "parallel_over_trees": cpu_par},

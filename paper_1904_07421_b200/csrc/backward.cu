@@ -93,7 +93,7 @@ __device__ __forceinline__ void store_tile(float (*S)[LDS_], int t, const float 
 // C[m, n] (+)= sum_k A(m, k) B(k, n), fp32.  A(m, k) = A[row(m) * lda + k] (A_ROW_M) or A[row(k) * lda + m];
 // B(k, n) = B[row(k) * ldb + n] (B_ROW_K) or B[n * ldb + k].
 template <bool A_ROW_M, bool B_ROW_K>
-__global__ void __launch_bounds__(GEMM_THREADS) sgemm_kernel(GemmArgs g) {
+__global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
     __shared__ __align__(16) float As[BK][LDS_];
     __shared__ __align__(16) float Bs[BK][LDS_];
     const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
