@@ -567,6 +567,11 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=device)
     jdb.lib()
 
+    if args.training_only:
+        flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=device)
+        wt = wl.make_workload(args.training_only, n_trees=args.trees)
+        print(json.dumps({"training": [time_training(args.training_only, wt, device, flush, args.steps, args.warmup)]}))
+        return
     pk = peaks()
     mode = {"auto": jdb.MODE_AUTO, "level": jdb.MODE_PER_LEVEL, "persistent": jdb.MODE_PERSISTENT}[args.mode]
     w = rank_workload(args.config, rank, args.trees)
@@ -689,6 +694,9 @@ def main():
     ap.add_argument("--all-configs", dest="all_configs", action="store_true", default=True,
                     help="also time the other four workloads and list them under per_config (1 GPU only)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
+    ap.add_argument("--training-only", type=int, default=0, choices=[0, 1, 2, 3, 4, 5],
+                    help="run only the training leg (fp32 forward + backward) of this workload and print its entry; "
+                         "for profiling the backward kernels (honours --trees, --steps, --warmup)")
     ap.add_argument("--rendezvous-only", action="store_true",
                     help="start the ranks, reduce the totals over gloo on the CPU and print them: checks the launcher, times nothing")
     args = ap.parse_args()

@@ -262,7 +262,8 @@ size_t jdb_treelstm_backward_workspace_bytes(int32_t n_nodes, int32_t n_edges, i
  *          zero); grad_c the same for c, or NULL for zeros.
  * dW [4H, D], dU [4H, H], db [4H]: outputs, dense, OVERWRITTEN (not accumulated).  dx [n_nodes, D] with leading
  * dimension lddx, or NULL to skip it.  The sums over nodes and edges behind dW, dU and db are split over CTAs whose
- * partial sums are added atomically: their last bits can differ from run to run.
+ * partial sums are added atomically, and so are the products of levels too small to fill the GPU otherwise: the last
+ * bits of every output can differ from run to run.
  * ws       device scratch of jdb_treelstm_backward_workspace_bytes bytes, 256-byte aligned.
  * Everything after the one synchronisation is asynchronous on `stream`; allocates nothing on the device. */
 jdb_status jdb_treelstm_backward(const jdb_forest *forest, const jdb_sched *sched, const float *x, int64_t ldx,

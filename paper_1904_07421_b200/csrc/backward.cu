@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
             if (gn >= g.N) continue;
             float v = acc[i][j];
             if (g.bias && blockIdx.z == 0) v += g.bias[gn];
-            if (ap) v += ap[gn];
+            if (ap && blockIdx.z == 0) v += ap[gn];
             if (atomic) atomicAdd(cp + gn, v);
             else if (g.beta) cp[gn] += v;
             else cp[gn] = v;
@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
 // ---- tables: edge slots in level order ------------------------------------------------------------------------------
 
 constexpr int SCAN_BLOCK = 1024;
+constexpr int SWEEP_STEPS = 2;   // least K steps per part when a level's GEMM is split to fill the SMs
 
 __device__ __forceinline__ int child_count(const int32_t* child_ptr, const int32_t* perm, int p, int n) {
     if (p >= n) return 0;
@@ -352,23 +353,30 @@ BwdWorkspace carve(void* ws, long long n, long long e, long long ni, int H) {
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+// min_steps: 0 = one CTA walks the whole contraction; else the contraction may be split over CTAs (partial sums added
+// atomically) as long as every part keeps at least that many K steps, until the launch has two CTAs per SM.  A split
+// result that is not accumulated (beta = 0) must be dense and is zeroed first.
 template <bool A_ROW_M, bool B_ROW_K>
-jdb_status gemm(GemmArgs g, bool split_k, int n_sm, cudaStream_t st) {
+jdb_status gemm(GemmArgs g, int min_steps, int n_sm, cudaStream_t st) {
     if (g.M <= 0 || g.N <= 0) return JDB_OK;
     g.vec_a = aligned16(g.A) && g.lda % 4 == 0;
     g.vec_b = aligned16(g.B) && g.ldb % 4 == 0;
     const int tm = ceil_div(g.M, BM), tn = ceil_div(g.N, BN);
     int splits = 1;
-    if (split_k) {   // enough CTAs for two per SM, every one with at least 16 K steps
+    if (min_steps > 0) {
         const long long tiles = (long long)tm * tn;
         const long long want = (2LL * n_sm + tiles - 1) / tiles;
-        const long long most = (g.K + 16 * BK - 1) / (16 * BK);
+        const long long most = (g.K + (long long)min_steps * BK - 1) / ((long long)min_steps * BK);
         splits = (int)(want < 1 ? 1 : (want > most ? most : want));
         if (splits < 1) splits = 1;
     }
     g.k_chunk = g.K <= 0 ? BK : ceil_div(ceil_div(g.K, splits), BK) * BK;
     splits = g.K <= 0 ? 1 : ceil_div(g.K, g.k_chunk);
     if (tn > 65535 || splits > 65535) return JDB_ERR_UNSUPPORTED;
+    if (splits > 1 && !g.beta) {
+        if (g.c_idx || g.ldc != g.N) return JDB_ERR_UNSUPPORTED;
+        JDB_CUDA_TRY(cudaMemsetAsync(g.C, 0, (size_t)g.M * g.N * sizeof(float), st));
+    }
     sgemm_kernel<A_ROW_M, B_ROW_K><<<dim3(tm, tn, splits), GEMM_THREADS, 0, st>>>(g);
     JDB_CUDA_TRY(cudaGetLastError());
     return JDB_OK;
@@ -400,7 +408,7 @@ jdb_status jdb_treelstm_backward(const jdb_forest* forest, const jdb_sched* sche
     if (!forest || !sched || forest->n_nodes < 0 || forest->n_edges < 0 || D <= 0 || H <= 0) return JDB_ERR_INVALID_ARG;
     if (!W || !U || !b || !dW || !dU || !db) return JDB_ERR_INVALID_ARG;
     const int n = forest->n_nodes, ne = forest->n_edges;
-    JDB_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)4 * H * D * sizeof(float), st));
+    JDB_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)4 * H * D * sizeof(float), st));   // zeroed here: also what an empty forest returns
     JDB_CUDA_TRY(cudaMemsetAsync(dU, 0, (size_t)4 * H * H * sizeof(float), st));
     JDB_CUDA_TRY(cudaMemsetAsync(db, 0, (size_t)4 * H * sizeof(float), st));
     if (n == 0) return JDB_OK;
@@ -446,18 +454,18 @@ jdb_status jdb_treelstm_backward(const jdb_forest* forest, const jdb_sched* sche
     {   // Z = x W^T + b for every node
         GemmArgs g{};
         g.A = x; g.lda = ldx; g.B = W; g.ldb = D; g.C = w.Z; g.ldc = 4LL * H; g.M = n; g.N = 4 * H; g.K = D; g.bias = b;
-        if ((s = gemm<true, false>(g, false, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return s;
     }
     if (ni > 0) {   // Z[internal, i o u] += h~ U_iou^T
         GemmArgs g{};
         g.A = w.HS; g.lda = H; g.B = U; g.ldb = H; g.C = w.Z; g.ldc = 4LL * H; g.M = ni; g.N = 3 * H; g.K = H;
         g.c_idx = perm + nl; g.beta = 1;
-        if ((s = gemm<true, false>(g, false, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return s;
     }
     if (ne > 0) {   // FE[slot] = U_f h_child
         GemmArgs g{};
         g.A = h; g.lda = ldh; g.a_idx = w.slot_child; g.B = U_f; g.ldb = H; g.C = w.FE; g.ldc = H; g.M = ne; g.N = H; g.K = H;
-        if ((s = gemm<true, false>(g, false, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return s;
     }
 
     for (int l = L - 1; l >= 0; --l) {
@@ -470,40 +478,43 @@ jdb_status jdb_treelstm_backward(const jdb_forest* forest, const jdb_sched* sche
         {   // DHS[r] = dz_iou(node at lo + r) U_iou: what every child of that node receives through the child sum
             GemmArgs g{};
             g.A = w.Z; g.lda = 4LL * H; g.a_idx = perm + lo; g.B = U; g.ldb = H; g.C = w.DHS; g.ldc = H; g.M = m; g.N = H; g.K = 3 * H;
-            if ((s = gemm<true, true>(g, false, n_sm, st)) != JDB_OK) return s;
+            if ((s = gemm<true, true>(g, SWEEP_STEPS, n_sm, st)) != JDB_OK) return s;
         }
         {   // dH[child] += dz_f(slot) U_f + DHS[parent]
             GemmArgs g{};
             g.A = w.FE + (size_t)e0 * H; g.lda = H; g.B = U_f; g.ldb = H; g.C = w.dH; g.ldc = H; g.M = e1 - e0; g.N = H; g.K = H;
             g.c_idx = w.slot_child + e0; g.beta = 1; g.add = w.DHS; g.add_idx = w.slot_ppos + e0; g.add_off = lo; g.ldadd = H;
-            if ((s = gemm<true, true>(g, false, n_sm, st)) != JDB_OK) return s;
+            if ((s = gemm<true, true>(g, SWEEP_STEPS, n_sm, st)) != JDB_OK) return s;
         }
     }
 
     {   // dW = dz^T x
         GemmArgs g{};
         g.A = w.Z; g.lda = 4LL * H; g.B = x; g.ldb = ldx; g.C = dW; g.ldc = D; g.M = 4 * H; g.N = D; g.K = n;
-        if ((s = gemm<false, true>(g, true, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<false, true>(g, 16, n_sm, st)) != JDB_OK) return s;
     }
     {
-        const int rows_per_block = 512;
+        // about four CTAs per SM, at least 32 rows each
+        const int col_blocks = ceil_div(4 * H, 128);
+        int rows_per_block = ceil_div(n, ceil_div(4 * n_sm, col_blocks));
+        if (rows_per_block < 32) rows_per_block = 32;
         column_sum_kernel<<<dim3(ceil_div(4 * H, 128), ceil_div(n, rows_per_block)), 128, 0, st>>>(w.Z, n, 4 * H, rows_per_block, db);
         JDB_CUDA_TRY(cudaGetLastError());
     }
     if (ni > 0) {   // dU_iou = dz_iou^T h~ over the internal nodes
         GemmArgs g{};
         g.A = w.Z; g.lda = 4LL * H; g.a_idx = perm + nl; g.B = w.HS; g.ldb = H; g.C = dU; g.ldc = H; g.M = 3 * H; g.N = H; g.K = ni;
-        if ((s = gemm<false, true>(g, true, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<false, true>(g, 16, n_sm, st)) != JDB_OK) return s;
     }
     if (ne > 0) {   // dU_f = sum over edges dz_f h_child^T
         GemmArgs g{};
         g.A = w.FE; g.lda = H; g.B = h; g.ldb = ldh; g.b_idx = w.slot_child; g.C = dU + (size_t)3 * H * H; g.ldc = H; g.M = H; g.N = H; g.K = ne;
-        if ((s = gemm<false, true>(g, true, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<false, true>(g, 16, n_sm, st)) != JDB_OK) return s;
     }
     if (dx) {   // dx = dz W
         GemmArgs g{};
         g.A = w.Z; g.lda = 4LL * H; g.B = W; g.ldb = D; g.C = dx; g.ldc = lddx; g.M = n; g.N = D; g.K = 4 * H;
-        if ((s = gemm<true, true>(g, false, n_sm, st)) != JDB_OK) return s;
+        if ((s = gemm<true, true>(g, lddx == D ? SWEEP_STEPS : 0, n_sm, st)) != JDB_OK) return s;
     }
     return JDB_OK;
 }
