@@ -39,6 +39,7 @@ struct GemmArgs {
     int beta;             // 1: C += result, 0: C = result
     int k_chunk;          // contraction range per blockIdx.z; more than one range: partial sums are added atomically
     int vec_a, vec_b;     // rows of A / B start on 16-byte boundaries and may be read four at a time
+    int tn;               // tiles along n
 };
 
 __device__ __forceinline__ float sigmoidf_(float v) { return 1.0f / (1.0f + expf(-v)); }
@@ -97,7 +98,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
     __shared__ __align__(16) float As[BK][LDS_];
     __shared__ __align__(16) float Bs[BK][LDS_];
     const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    // tiles that share rows of A are neighbours in the grid: A reaches DRAM once, B (the smaller operand) stays in L2
+    const int m0 = (blockIdx.x / g.tn) * BM, n0 = (blockIdx.x % g.tn) * BN;
     const int kbeg = blockIdx.z * g.k_chunk;
     const int kend = min(g.K, kbeg + g.k_chunk);
     float acc[8][8];
@@ -362,22 +364,27 @@ jdb_status gemm(GemmArgs g, int min_steps, int n_sm, cudaStream_t st) {
     g.vec_a = aligned16(g.A) && g.lda % 4 == 0;
     g.vec_b = aligned16(g.B) && g.ldb % 4 == 0;
     const int tm = ceil_div(g.M, BM), tn = ceil_div(g.N, BN);
+    const long long tiles = (long long)tm * tn;
     int splits = 1;
-    if (min_steps > 0) {
-        const long long tiles = (long long)tm * tn;
-        const long long want = (2LL * n_sm + tiles - 1) / tiles;
+    if (min_steps > 0 && tiles < 2LL * n_sm) {
+        // the number of parts that fills whole waves of two CTAs per SM best (fewest parts among equals)
         const long long most = (g.K + (long long)min_steps * BK - 1) / ((long long)min_steps * BK);
-        splits = (int)(want < 1 ? 1 : (want > most ? most : want));
-        if (splits < 1) splits = 1;
+        double best = 0.0;
+        for (long long sp = 1; sp <= most && sp <= 64; ++sp) {
+            const long long ctas = tiles * sp, waves = (ctas + 2 * n_sm - 1) / (2 * n_sm);
+            const double fill = (double)ctas / (double)(waves * 2 * n_sm);
+            if (fill > best + 0.02) { best = fill; splits = (int)sp; }
+        }
     }
     g.k_chunk = g.K <= 0 ? BK : ceil_div(ceil_div(g.K, splits), BK) * BK;
     splits = g.K <= 0 ? 1 : ceil_div(g.K, g.k_chunk);
-    if (tn > 65535 || splits > 65535) return JDB_ERR_UNSUPPORTED;
+    if (tiles > 0x7fffffffLL || splits > 65535) return JDB_ERR_UNSUPPORTED;
+    g.tn = tn;
     if (splits > 1 && !g.beta) {
         if (g.c_idx || g.ldc != g.N) return JDB_ERR_UNSUPPORTED;
         JDB_CUDA_TRY(cudaMemsetAsync(g.C, 0, (size_t)g.M * g.N * sizeof(float), st));
     }
-    sgemm_kernel<A_ROW_M, B_ROW_K><<<dim3(tm, tn, splits), GEMM_THREADS, 0, st>>>(g);
+    sgemm_kernel<A_ROW_M, B_ROW_K><<<dim3((unsigned)tiles, 1, splits), GEMM_THREADS, 0, st>>>(g);
     JDB_CUDA_TRY(cudaGetLastError());
     return JDB_OK;
 }
