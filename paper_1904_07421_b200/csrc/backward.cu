@@ -321,9 +321,14 @@ __global__ void column_sum_kernel(const float* __restrict__ Z, int n, int cols, 
     const int col = blockIdx.x * blockDim.x + threadIdx.x;
     if (col >= cols) return;
     const int r0 = blockIdx.y * rows_per_block, r1 = min(n, r0 + rows_per_block);
-    float s = 0.0f;
-    for (int r = r0; r < r1; ++r) s += Z[(long long)r * cols + col];
-    atomicAdd(out + col, s);
+    float s[4] = {0.0f, 0.0f, 0.0f, 0.0f};   // four loads in flight per thread
+    int r = r0;
+    for (; r + 4 <= r1; r += 4) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) s[q] += Z[(long long)(r + q) * cols + col];
+    }
+    for (; r < r1; ++r) s[0] += Z[(long long)r * cols + col];
+    atomicAdd(out + col, (s[0] + s[1]) + (s[2] + s[3]));
 }
 
 // ---- host -----------------------------------------------------------------------------------------------------------
@@ -501,9 +506,9 @@ jdb_status jdb_treelstm_backward(const jdb_forest* forest, const jdb_sched* sche
         if ((s = gemm<false, true>(g, 16, n_sm, st)) != JDB_OK) return s;
     }
     {
-        // about four CTAs per SM, at least 32 rows each
+        // about 32 CTAs of 128 threads per SM, at least 32 rows each
         const int col_blocks = ceil_div(4 * H, 128);
-        int rows_per_block = ceil_div(n, ceil_div(4 * n_sm, col_blocks));
+        int rows_per_block = ceil_div(n, ceil_div(32 * n_sm, col_blocks));
         if (rows_per_block < 32) rows_per_block = 32;
         column_sum_kernel<<<dim3(ceil_div(4 * H, 128), ceil_div(n, rows_per_block)), 128, 0, st>>>(w.Z, n, 4 * H, rows_per_block, db);
         JDB_CUDA_TRY(cudaGetLastError());
