@@ -15,154 +15,14 @@
 #include <vector>
 
 #include "common.cuh"
+#include "scan.cuh"
+#include "sgemm.cuh"
 
 namespace jdb {
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 16, GEMM_THREADS = 256;
-constexpr int LDS_ = BM + 4;   // row pitch of a staged tile (floats): keeps 16-byte alignment of the 4-wide reads
-
-struct GemmArgs {
-    const float* A;
-    const float* B;
-    float* C;
-    long long lda, ldb, ldc;
-    int M, N, K;
-    const int* a_idx;     // row gather of A: along m (A_ROW_M) or along k
-    const int* b_idx;     // row gather of B along k (B_ROW_K only)
-    const int* c_idx;     // row scatter of C
-    const float* bias;    // [N] added to every row (null = none)
-    const float* add;     // rows added to the result: add[(add_idx[m] - add_off) * ldadd + n] (null = none)
-    const int* add_idx;
-    int add_off;
-    long long ldadd;
-    int beta;             // 1: C += result, 0: C = result
-    int k_chunk;          // contraction range per blockIdx.z; more than one range: partial sums are added atomically
-    int vec_a, vec_b;     // rows of A / B start on 16-byte boundaries and may be read four at a time
-    int tn;               // tiles along n
-};
-
-__device__ __forceinline__ float sigmoidf_(float v) { return 1.0f / (1.0f + expf(-v)); }
-
-// Eight elements of a tile for this thread.  ROW_MN: the matrix row is the tile's m (or n) index and k runs along it
-// (thread: row t / 2, eight k from (t % 2) * 8); else the matrix row is k and m (or n) runs along it (thread: k = t / 16,
-// eight m from (t % 16) * 8).
-template <bool ROW_MN>
-__device__ __forceinline__ void load_tile(const float* __restrict__ base, long long ld, const int* __restrict__ idx, int mn0,
-                                          int MN, int k0, int kend, int vec, int t, float (&r)[8]) {
-    int row, along0, along_end;
-    bool row_ok;
-    if (ROW_MN) {
-        const int g = mn0 + (t >> 1);
-        row_ok = g < MN;
-        row = row_ok ? (idx ? idx[g] : g) : 0;
-        along0 = k0 + (t & 1) * 8;
-        along_end = kend;
-    } else {
-        const int g = k0 + (t >> 4);
-        row_ok = g < kend;
-        row = row_ok ? (idx ? idx[g] : g) : 0;
-        along0 = mn0 + (t & 15) * 8;
-        along_end = MN;
-    }
-    const float* p = base + (long long)row * ld + along0;
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        if (row_ok && vec && along0 + 4 * q + 4 <= along_end) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p + 4 * q));
-            r[4 * q] = v.x; r[4 * q + 1] = v.y; r[4 * q + 2] = v.z; r[4 * q + 3] = v.w;
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) r[4 * q + i] = (row_ok && along0 + 4 * q + i < along_end) ? __ldg(p + 4 * q + i) : 0.0f;
-        }
-    }
-}
-
-template <bool ROW_MN>
-__device__ __forceinline__ void store_tile(float (*S)[LDS_], int t, const float (&r)[8]) {
-    if (ROW_MN) {
-        const int mn = t >> 1, k = (t & 1) * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) S[k + i][mn] = r[i];
-    } else {
-        const int k = t >> 4, mn = (t & 15) * 8;
-        *reinterpret_cast<float4*>(&S[k][mn]) = make_float4(r[0], r[1], r[2], r[3]);
-        *reinterpret_cast<float4*>(&S[k][mn + 4]) = make_float4(r[4], r[5], r[6], r[7]);
-    }
-}
-
-// C[m, n] (+)= sum_k A(m, k) B(k, n), fp32.  A(m, k) = A[row(m) * lda + k] (A_ROW_M) or A[row(k) * lda + m];
-// B(k, n) = B[row(k) * ldb + n] (B_ROW_K) or B[n * ldb + k].
-template <bool A_ROW_M, bool B_ROW_K>
-__global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
-    __shared__ __align__(16) float As[BK][LDS_];
-    __shared__ __align__(16) float Bs[BK][LDS_];
-    const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
-    // tiles that share rows of A are neighbours in the grid: A reaches DRAM once, B (the smaller operand) stays in L2
-    const int m0 = (blockIdx.x / g.tn) * BM, n0 = (blockIdx.x % g.tn) * BN;
-    const int kbeg = blockIdx.z * g.k_chunk;
-    const int kend = min(g.K, kbeg + g.k_chunk);
-    float acc[8][8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
-
-    float ra[8], rb[8];
-    if (kbeg < kend) {
-        load_tile<A_ROW_M>(g.A, g.lda, g.a_idx, m0, g.M, kbeg, kend, g.vec_a, t, ra);
-        load_tile<!B_ROW_K>(g.B, g.ldb, g.b_idx, n0, g.N, kbeg, kend, g.vec_b, t, rb);
-    }
-    for (int k0 = kbeg; k0 < kend; k0 += BK) {
-        store_tile<A_ROW_M>(As, t, ra);
-        store_tile<!B_ROW_K>(Bs, t, rb);
-        __syncthreads();
-        if (k0 + BK < kend) {   // the next tile's loads fly while this one is multiplied
-            load_tile<A_ROW_M>(g.A, g.lda, g.a_idx, m0, g.M, k0 + BK, kend, g.vec_a, t, ra);
-            load_tile<!B_ROW_K>(g.B, g.ldb, g.b_idx, n0, g.N, k0 + BK, kend, g.vec_b, t, rb);
-        }
-#pragma unroll
-        for (int k = 0; k < BK; ++k) {
-            const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
-            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
-            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-    if (kbeg >= kend && blockIdx.z > 0) return;
-
-    const bool atomic = gridDim.z > 1;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
-        if (gm >= g.M) continue;
-        const long long crow = g.c_idx ? g.c_idx[gm] : gm;
-        float* cp = g.C + crow * g.ldc;
-        const float* ap = g.add ? g.add + (long long)(g.add_idx[gm] - g.add_off) * g.ldadd : nullptr;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int gn = n0 + (j < 4 ? tx * 4 + j : 64 + tx * 4 + (j - 4));
-            if (gn >= g.N) continue;
-            float v = acc[i][j];
-            if (g.bias && blockIdx.z == 0) v += g.bias[gn];
-            if (ap && blockIdx.z == 0) v += ap[gn];
-            if (atomic) atomicAdd(cp + gn, v);
-            else if (g.beta) cp[gn] += v;
-            else cp[gn] = v;
-        }
-    }
-}
-
 // ---- tables: edge slots in level order ------------------------------------------------------------------------------
 
-constexpr int SCAN_BLOCK = 1024;
 constexpr int SWEEP_STEPS = 2;   // least K steps per part when a level's GEMM is split to fill the SMs
 
 __device__ __forceinline__ int child_count(const int32_t* child_ptr, const int32_t* perm, int p, int n) {
@@ -171,57 +31,11 @@ __device__ __forceinline__ int child_count(const int32_t* child_ptr, const int32
     return child_ptr[j + 1] - child_ptr[j];
 }
 
-// exclusive scan of one value per thread over a block of SCAN_BLOCK threads; returns the thread's offset, total in `total`
-__device__ __forceinline__ int block_exclusive_scan(int v, int& total) {
-    __shared__ int warp_sum[32];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    int incl = v;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int o = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += o;
-    }
-    if (lane == 31) warp_sum[w] = incl;
-    __syncthreads();
-    if (w == 0) {
-        int s = warp_sum[lane];
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int o = __shfl_up_sync(0xffffffffu, s, d);
-            if (lane >= d) s += o;
-        }
-        warp_sum[lane] = s;
-    }
-    __syncthreads();
-    total = warp_sum[31];
-    const int before = w > 0 ? warp_sum[w - 1] : 0;
-    __syncthreads();
-    return before + incl - v;
-}
-
 __global__ void __launch_bounds__(SCAN_BLOCK) slot_count_kernel(const int32_t* child_ptr, const int32_t* perm, int n, int* block_sum) {
     const int p = blockIdx.x * SCAN_BLOCK + threadIdx.x;
     int total;
     block_exclusive_scan(child_count(child_ptr, perm, p, n), total);
     if (threadIdx.x == 0) block_sum[blockIdx.x] = total;
-}
-
-// one CTA turns the block sums into block offsets (in place)
-__global__ void __launch_bounds__(SCAN_BLOCK) slot_scan_kernel(int* block_sum, int n_blocks) {
-    __shared__ int carry;
-    if (threadIdx.x == 0) carry = 0;
-    __syncthreads();
-    for (int b0 = 0; b0 < n_blocks; b0 += SCAN_BLOCK) {
-        const int i = b0 + threadIdx.x;
-        const int v = i < n_blocks ? block_sum[i] : 0;
-        int total;
-        const int off = block_exclusive_scan(v, total);
-        const int base = carry;
-        if (i < n_blocks) block_sum[i] = base + off;
-        __syncthreads();
-        if (threadIdx.x == 0) carry = base + total;
-        __syncthreads();
-    }
 }
 
 // edge_ptr[p] = edge slots before position p; per slot: the child's node id and the parent's position
@@ -358,42 +172,6 @@ BwdWorkspace carve(void* ws, long long n, long long e, long long ni, int H) {
     return w;
 }
 
-bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
-
-// min_steps: 0 = one CTA walks the whole contraction; else the contraction may be split over CTAs (partial sums added
-// atomically) as long as every part keeps at least that many K steps, until the launch has two CTAs per SM.  A split
-// result that is not accumulated (beta = 0) must be dense and is zeroed first.
-template <bool A_ROW_M, bool B_ROW_K>
-jdb_status gemm(GemmArgs g, int min_steps, int n_sm, cudaStream_t st) {
-    if (g.M <= 0 || g.N <= 0) return JDB_OK;
-    g.vec_a = aligned16(g.A) && g.lda % 4 == 0;
-    g.vec_b = aligned16(g.B) && g.ldb % 4 == 0;
-    const int tm = ceil_div(g.M, BM), tn = ceil_div(g.N, BN);
-    const long long tiles = (long long)tm * tn;
-    int splits = 1;
-    if (min_steps > 0 && tiles < 2LL * n_sm) {
-        // the number of parts that fills whole waves of two CTAs per SM best (fewest parts among equals)
-        const long long most = (g.K + (long long)min_steps * BK - 1) / ((long long)min_steps * BK);
-        double best = 0.0;
-        for (long long sp = 1; sp <= most && sp <= 64; ++sp) {
-            const long long ctas = tiles * sp, waves = (ctas + 2 * n_sm - 1) / (2 * n_sm);
-            const double fill = (double)ctas / (double)(waves * 2 * n_sm);
-            if (fill > best + 0.02) { best = fill; splits = (int)sp; }
-        }
-    }
-    g.k_chunk = g.K <= 0 ? BK : ceil_div(ceil_div(g.K, splits), BK) * BK;
-    splits = g.K <= 0 ? 1 : ceil_div(g.K, g.k_chunk);
-    if (tiles > 0x7fffffffLL || splits > 65535) return JDB_ERR_UNSUPPORTED;
-    g.tn = tn;
-    if (splits > 1 && !g.beta) {
-        if (g.c_idx || g.ldc != g.N) return JDB_ERR_UNSUPPORTED;
-        JDB_CUDA_TRY(cudaMemsetAsync(g.C, 0, (size_t)g.M * g.N * sizeof(float), st));
-    }
-    sgemm_kernel<A_ROW_M, B_ROW_K><<<dim3((unsigned)tiles, 1, splits), GEMM_THREADS, 0, st>>>(g);
-    JDB_CUDA_TRY(cudaGetLastError());
-    return JDB_OK;
-}
-
 }  // namespace
 
 size_t backward_ws_bytes(int32_t n_nodes, int32_t n_edges, int32_t n_internal_bound, int32_t H) {
@@ -440,7 +218,7 @@ jdb_status jdb_treelstm_backward(const jdb_forest* forest, const jdb_sched* sche
     // edge slots in level order and the level table on the host
     const int n_blocks = n / SCAN_BLOCK + 1;   // covers position n too (the total)
     slot_count_kernel<<<n_blocks, SCAN_BLOCK, 0, st>>>(forest->child_ptr, perm, n, w.block_sum);
-    slot_scan_kernel<<<1, SCAN_BLOCK, 0, st>>>(w.block_sum, n_blocks);
+    block_sums_scan_kernel<<<1, SCAN_BLOCK, 0, st>>>(w.block_sum, n_blocks);
     slot_fill_kernel<<<n_blocks, SCAN_BLOCK, 0, st>>>(forest->child_ptr, forest->child_idx, perm, n, ne, w.block_sum, w.edge_ptr,
                                                      w.slot_child, w.slot_ppos);
     level_table_kernel<<<ceil_div(L + 1, 256), 256, 0, st>>>(sched->level_ptr, w.edge_ptr, L, w.lv);
