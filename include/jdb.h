@@ -272,6 +272,60 @@ jdb_status jdb_treelstm_backward(const jdb_forest *forest, const jdb_sched *sche
                                  float *dW, float *dU, float *db, float *dx, int64_t lddx, void *ws, size_t ws_bytes,
                                  void *stream);
 
+/* ---- nodes of several kinds: the table keyed by (depth, key) and its execution (Sections 4.2 and 4.3) ---------- */
+
+/* Section 4.2 files every node under its depth and a key made of its type, its settings and the layout of its
+ * arguments; nodes that share both share a slot, and the slots run in depth order, one batched launch each
+ * (Section 4.3).  Here `key[v]` (0 .. n_keys-1) stands for that triple: equal keys are batchable with each other.
+ * All arrays are caller-allocated device memory. */
+typedef struct {
+    int32_t *perm;       /* [n_nodes] node ids ordered by (depth, key, id)                                  */
+    int32_t *slot_ptr;   /* [n_nodes + 1] capacity; entries 0..n_slots valid: first position of every slot  */
+    int32_t *slot_depth; /* [n_nodes] capacity; depth of the nodes of slot s                                */
+    int32_t *slot_key;   /* [n_nodes] capacity; their key                                                   */
+    int32_t n_slots;     /* host; written by jdb_batch_plan                                                 */
+    int32_t bad_key;     /* host; 1 if some key lay outside 0 .. n_keys-1 (it was filed as key 0)           */
+} jdb_plan;
+
+size_t jdb_batch_plan_workspace_bytes(int32_t n_nodes);
+
+/* Builds the table from the depths of a schedule made by jdb_schedule on `forest` (its level count bounds the sort
+ * key; n_levels * n_keys must stay below 2^31, else JDB_ERR_UNSUPPORTED).  Synchronises `stream` once to read back the
+ * slot count.  A key out of range gives JDB_ERR_INVALID_ARG (the table is still complete, with that key taken as 0).
+ * n_nodes = 0 gives n_slots = 0 and slot_ptr[0] = 0.  ws: device scratch, 256-byte aligned. */
+jdb_status jdb_batch_plan(const jdb_forest *forest, const jdb_sched *sched, const int32_t *key, int32_t n_keys,
+                          jdb_plan *out, void *ws, size_t ws_bytes, void *stream);
+
+/* One kind of cell with its own parameters (the "same parameterisation" condition of Section 1: nodes batch only with
+ * nodes of the same cell).  W [4H, D], b [4H] in row blocks (i, o, u, f), fp32 row-major device arrays.
+ * JDB_CELL_CHILDSUM: the cell of jdb_treelstm_forward, U [4H, H], any number of children.
+ * JDB_CELL_NARY: the N-ary Tree-LSTM cell of the same cited model, one recurrent matrix per child position:
+ *     (i, o, u) = (sig, sig, tanh)(W x + sum_l U^l h_l + b);  f_k = sig(W_f x + sum_l U_f^kl h_l + b_f);
+ *     c = i*u + sum_k f_k*c_k;  h = o*tanh(c);
+ *   U [(3 + arity) H, arity H]: row blocks (i, o, u, f_1 .. f_arity), column block l multiplies child l's h; a node
+ *   with fewer children than `arity` (1 .. 8) treats the missing ones as zero states, one with more is an error. */
+enum { JDB_CELL_CHILDSUM = 0, JDB_CELL_NARY = 1 };
+typedef struct {
+    int32_t kind;   /* JDB_CELL_* */
+    int32_t arity;  /* JDB_CELL_NARY: child positions; ignored for JDB_CELL_CHILDSUM */
+    const float *W;
+    const float *U;
+    const float *b;
+} jdb_cell;
+
+size_t jdb_cells_forward_workspace_bytes(int32_t n_nodes, int32_t n_edges, int32_t H, int32_t max_arity, int32_t n_keys);
+
+/* Runs the table: for every slot in order, the cell `cells[slot_key]` over the slot's nodes as one batch (fp32 on the
+ * CUDA cores: W x + b of the slot's rows, the recurrent products of the cell's kind, then its pointwise part).
+ * cells    HOST array of n_keys descriptors (their W, U, b are device pointers).
+ * key      the array given to jdb_batch_plan.  x [n_nodes, D] fp32 (ldx); h, c [n_nodes, H] fp32 outputs (ldh).
+ * Copies the slot table to the host and synchronises `stream` once before its launches; a node with more children
+ * than its cell's arity, or a plan that does not fit the forest's totals, gives JDB_ERR_INVALID_ARG.  Allocates nothing
+ * on the device.  ws: device scratch of jdb_cells_forward_workspace_bytes bytes, 256-byte aligned. */
+jdb_status jdb_cells_forward(const jdb_forest *forest, const jdb_plan *plan, const int32_t *key, const jdb_cell *cells,
+                             int32_t n_keys, const float *x, int64_t ldx, int32_t D, int32_t H, float *h, float *c,
+                             int64_t ldh, void *ws, size_t ws_bytes, void *stream);
+
 /* ---- one call from host buffers (what a user without device arrays calls) -------------------- */
 
 /* Device scratch needed by jdb_treelstm_forward_host (CSR, x, schedule, h, c and both workspaces). */

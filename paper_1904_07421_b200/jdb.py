@@ -30,7 +30,9 @@ EXPORTS = [
     "jdb_treelstm_forward", "jdb_sched_status", "jdb_debug_report", "jdb_forward_host_workspace_bytes",
     "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts", "jdb_relatedness_head",
     "jdb_treelstm_backward_workspace_bytes", "jdb_treelstm_backward",
+    "jdb_batch_plan_workspace_bytes", "jdb_batch_plan", "jdb_cells_forward_workspace_bytes", "jdb_cells_forward",
 ]
+CELL_CHILDSUM, CELL_NARY = 0, 1
 
 
 class CForest(C.Structure):
@@ -107,6 +109,14 @@ def lib():
     L.jdb_treelstm_backward.restype = C.c_int
     L.jdb_treelstm_backward.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, i32, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, i64,
                                         vp, C.c_size_t, vp]
+    L.jdb_batch_plan_workspace_bytes.restype = C.c_size_t
+    L.jdb_batch_plan_workspace_bytes.argtypes = [i32]
+    L.jdb_batch_plan.restype = C.c_int
+    L.jdb_batch_plan.argtypes = [vp, vp, vp, i32, vp, vp, C.c_size_t, vp]
+    L.jdb_cells_forward_workspace_bytes.restype = C.c_size_t
+    L.jdb_cells_forward_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    L.jdb_cells_forward.restype = C.c_int
+    L.jdb_cells_forward.argtypes = [vp, vp, vp, vp, i32, vp, i64, i32, i32, vp, vp, i64, vp, C.c_size_t, vp]
     L.jdb_relatedness_head.restype = C.c_int
     L.jdb_relatedness_head.argtypes = [vp, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
@@ -333,6 +343,70 @@ def jdb_treelstm_backward(forest: Forest, sched: Schedule, x: torch.Tensor, W: t
     if st != OK:
         raise JdbError(st, "jdb_treelstm_backward")
     return dW, dU, db, (dx[:n] if want_dx else None)
+
+
+class CPlan(C.Structure):
+    _fields_ = [("perm", C.c_void_p), ("slot_ptr", C.c_void_p), ("slot_depth", C.c_void_p), ("slot_key", C.c_void_p),
+                ("n_slots", C.c_int32), ("bad_key", C.c_int32)]
+
+
+class CCell(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("arity", C.c_int32), ("W", C.c_void_p), ("U", C.c_void_p), ("b", C.c_void_p)]
+
+
+@dataclass
+class Plan:
+    perm: torch.Tensor        # int32 [n_nodes]: node ids by (depth, key, id)
+    slot_ptr: torch.Tensor    # int32, entries 0..n_slots valid
+    slot_depth: torch.Tensor
+    slot_key: torch.Tensor
+    n_slots: int = 0
+
+    def c(self) -> CPlan:
+        return CPlan(self.perm.data_ptr(), self.slot_ptr.data_ptr(), self.slot_depth.data_ptr(), self.slot_key.data_ptr(),
+                     self.n_slots, 0)
+
+
+def jdb_batch_plan(forest: Forest, sched: Schedule, key: torch.Tensor, n_keys: int, stream=None) -> Plan:
+    """The table of Section 4.2 for nodes of several kinds: slots by (depth, key), ids ascending inside a slot."""
+    dev = forest.child_ptr.device
+    n = max(forest.n_nodes, 1)
+    mk = lambda k: torch.empty(k, dtype=torch.int32, device=dev)
+    out = Plan(mk(n), mk(n + 1), mk(n), mk(n))
+    key = key.to(torch.int32).contiguous()
+    ws = _device_bytes(lib().jdb_batch_plan_workspace_bytes(forest.n_nodes), dev)
+    cf, cs, cp = forest.c(), sched.c(), out.c()
+    st = lib().jdb_batch_plan(C.byref(cf), C.byref(cs), _ptr(key), n_keys, C.byref(cp), _ptr(ws), ws.numel(), _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_batch_plan")
+    out.n_slots = cp.n_slots
+    return out
+
+
+def jdb_cells_forward(forest: Forest, plan: Plan, key: torch.Tensor, cells, x: torch.Tensor, D: int, H: int,
+                      h: Optional[torch.Tensor] = None, c: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                      stream=None):
+    """h, c [n_nodes, H] fp32 of a forest whose node v is a cell of kind cells[key[v]].
+
+    cells: list of (kind, arity, W, U, b) with fp32 device tensors (kind CELL_CHILDSUM or CELL_NARY).
+    """
+    dev = forest.child_ptr.device
+    n = max(forest.n_nodes, 1)
+    h = torch.empty((n, H), dtype=torch.float32, device=dev) if h is None else h
+    c = torch.empty((n, H), dtype=torch.float32, device=dev) if c is None else c
+    key = key.to(torch.int32).contiguous()
+    keep = [tuple(t.to(torch.float32).contiguous() for t in cell[2:5]) for cell in cells]   # alive until the call returns
+    arr = (CCell * len(cells))(*[CCell(int(cell[0]), int(cell[1]), W.data_ptr(), U.data_ptr(), b.data_ptr())
+                                 for cell, (W, U, b) in zip(cells, keep)])
+    amax = max([int(cell[1]) for cell in cells if int(cell[0]) == CELL_NARY] + [0])
+    if ws is None:
+        ws = _device_bytes(lib().jdb_cells_forward_workspace_bytes(forest.n_nodes, forest.n_edges, H, amax, len(cells)), dev)
+    cf, cp = forest.c(), plan.c()
+    st = lib().jdb_cells_forward(C.byref(cf), C.byref(cp), _ptr(key), arr, len(cells), _ptr(x), x.stride(0) if forest.n_nodes else D,
+                                 D, H, _ptr(h), _ptr(c), h.stride(0), _ptr(ws), ws.numel(), _stream(stream))
+    if st != OK:
+        raise JdbError(st, "jdb_cells_forward")
+    return h[:forest.n_nodes], c[:forest.n_nodes]
 
 
 def jdb_debug_report(sched: Schedule, stream=None):
