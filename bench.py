@@ -511,6 +511,55 @@ def time_training(idx: int, w: wl.Workload, device, flush, steps: int = 5, warmu
             "launches_backward": 4 + 2 + 3 + 3 * max(sched.n_levels - 1, 0) + 1 + 5}
 
 
+def time_batcher(idx: int, w: wl.Workload, device, flush, steps: int = 5, warmup: int = 3):
+    """Section 4.2's table for nodes of two kinds (a Child-Sum and an N-ary cell drawn per node) and its execution slot
+    by slot in fp32: jdb_batch_plan + jdb_cells_forward on the workload's forest.  Not part of `value`."""
+    import torch
+    from paper_1904_07421_b200 import jdb
+    f = w.forest
+    D, H = w.D, w.H
+    rng = np.random.default_rng(13)
+    kids = np.diff(f.child_ptr)
+    arity = int(max(1, kids.max()))
+    if arity > 8:
+        return None
+    key_h = rng.integers(0, 2, size=f.n_nodes).astype(np.int32)
+    forest = jdb.forest_to_device(f.child_ptr, f.child_idx, device)
+    x = torch.from_numpy(w.x_full()).to(device)
+    Un = (rng.standard_normal(((3 + arity) * H, arity * H)) / np.sqrt(arity * H)).astype(np.float32)
+    cells = [(jdb.CELL_CHILDSUM, 0, *(torch.from_numpy(a).to(device) for a in (w.W, w.U, w.b))),
+             (jdb.CELL_NARY, arity, *(torch.from_numpy(a).to(device) for a in (w.W, Un, w.b)))]
+    key = torch.from_numpy(key_h).to(device)
+    sched = jdb.jdb_schedule(forest)
+    h = torch.empty((f.n_nodes, H), dtype=torch.float32, device=device)
+    c = torch.empty_like(h)
+    ws = torch.empty(jdb.lib().jdb_cells_forward_workspace_bytes(f.n_nodes, f.n_edges, H, arity, 2), dtype=torch.uint8, device=device)
+    t_plan, t_run = [], []
+    plan = None
+    for it in range(warmup + steps):
+        flush.add_(1)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        plan = jdb.jdb_batch_plan(forest, sched, key, 2)
+        e[1].record()
+        jdb.jdb_cells_forward(forest, plan, key, cells, x, D, H, h=h, c=c, ws=ws)
+        e[2].record()
+        e[2].synchronize()
+        if it >= warmup:
+            t_plan.append(e[0].elapsed_time(e[1]))
+            t_run.append(e[1].elapsed_time(e[2]))
+    tp, tr = statistics.median(t_plan), statistics.median(t_run)
+    internal = kids > 0
+    flops = (8.0 * f.n_nodes * D * H
+             + float(np.sum((6.0 + 2.0 * kids) * H * H * (internal & (key_h == 0))))
+             + float(np.sum(2.0 * (3 + arity) * kids * H * H * (internal & (key_h == 1)))))
+    return {"config": idx, "workload": w.name, "nodes": f.n_nodes, "levels": int(sched.n_levels), "slots": int(plan.n_slots),
+            "cells": ["childsum", f"nary(arity {arity})"], "D": D, "H": H, "dtype": "f32",
+            "step": "jdb_batch_plan + jdb_cells_forward", "plan_ms": tp, "forward_ms": tr,
+            "nodes_per_s": f.n_nodes / ((tp + tr) * 1e-3), "flops": flops, "tflops": flops / (tr * 1e-3) / 1e12,
+            "frac_of_fp32_alu_peak": flops / (tr * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS}
+
+
 def rank_workload(config: int, rank: int, n_trees=None) -> wl.Workload:
     """Every rank draws its own forest of the workload's shape (weak scaling over independent trees)."""
     return wl.make_workload(config, n_trees=n_trees, seed=None if rank == 0 else wl.BASE_SEED + config + 1000 * rank)
@@ -570,7 +619,8 @@ def run_gpu(args):
     if args.training_only:
         flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=device)
         wt = wl.make_workload(args.training_only, n_trees=args.trees)
-        print(json.dumps({"training": [time_training(args.training_only, wt, device, flush, args.steps, args.warmup)]}))
+        print(json.dumps({"training": [time_training(args.training_only, wt, device, flush, args.steps, args.warmup)],
+                          "keyed_batcher": [time_batcher(args.training_only, wt, device, flush, args.steps, args.warmup)]}))
         return
     pk = peaks()
     mode = {"auto": jdb.MODE_AUTO, "level": jdb.MODE_PER_LEVEL, "persistent": jdb.MODE_PERSISTENT}[args.mode]
@@ -626,10 +676,15 @@ def run_gpu(args):
                 per_config.append(config_entry(idx, wi, ji, ti, args.steps, wi.forest.n_nodes * args.steps / (sum(ti) / 1e3), ri, pf, po))
                 del ji, wi
                 torch.cuda.empty_cache()
-        training = []
+        training, batcher = [], []
         if args.all_configs and world == 1:
             for idx in (1, 2, 3, 4):
                 training.append(time_training(idx, wl.make_workload(idx), device, flush))
+                torch.cuda.empty_cache()
+            for idx in (1, 2, 3):
+                b = time_batcher(idx, wl.make_workload(idx), device, flush)
+                if b is not None:
+                    batcher.append(b)
                 torch.cuda.empty_cache()
         cpu_v, cpu_sample, cpu_trees = time_oracle(w, args.cpu_budget)
         cpu_par = None
@@ -655,6 +710,7 @@ def run_gpu(args):
             "phases": phases_out,
             "relatedness_head": head,
             "training": training,
+            "keyed_batcher": batcher,
             "batching_ratio": f.n_nodes / max(n_levels_main, 1),   # cells evaluated per batched step: Section 3's batching ratio at cell granularity
             "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample,
                              "parallel_over_trees": cpu_par},

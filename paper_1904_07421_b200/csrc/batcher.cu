@@ -151,6 +151,8 @@ __global__ void __launch_bounds__(SCAN_BLOCK) slot_start_fill_kernel(const int32
 
 // ---- execution ------------------------------------------------------------------------------------------------------
 
+constexpr int SLOT_STEPS = 2;   // least K steps per part when a slot's product is split to fill the SMs
+
 // kid[l * n + p] = child l of the node at plan position p, or -1; *bad = 1 if an N-ary node has more children than its arity
 __global__ void child_positions_kernel(const int32_t* __restrict__ child_ptr, const int32_t* __restrict__ child_idx,
                                        const int32_t* __restrict__ perm, const int32_t* __restrict__ key, const int32_t* __restrict__ arity_of,
@@ -163,6 +165,40 @@ __global__ void child_positions_kernel(const int32_t* __restrict__ child_ptr, co
     const int e0 = child_ptr[j], cnt = child_ptr[j + 1] - e0;
     if (a > 0 && cnt > a) *bad = 1;
     for (int l = 0; l < amax; ++l) kid[(size_t)l * n + p] = (a > 0 && l < cnt && l < a) ? child_idx[e0 + l] : -1;
+}
+
+// Rows that have a child in position l, compacted in plan order (most nodes of an N-ary cell have fewer children
+// than the arity, and a product over a position should not pay for the rows that have no child there):
+// cptr[p] = such rows before position p; ckid / cpos = the child's node id and the row's position.
+__global__ void __launch_bounds__(SCAN_BLOCK) position_count_kernel(const int32_t* __restrict__ kid_l, int n, int* block_sum) {
+    const int p = blockIdx.x * SCAN_BLOCK + threadIdx.x;
+    int total;
+    block_exclusive_scan((p < n && kid_l[p] >= 0) ? 1 : 0, total);
+    if (threadIdx.x == 0) block_sum[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(SCAN_BLOCK) position_fill_kernel(const int32_t* __restrict__ kid_l, int n, const int* block_off,
+                                                                   int32_t* __restrict__ cptr, int32_t* __restrict__ ckid,
+                                                                   int32_t* __restrict__ cpos) {
+    const int p = blockIdx.x * SCAN_BLOCK + threadIdx.x;
+    const int flag = (p < n && kid_l[p] >= 0) ? 1 : 0;
+    int total;
+    const int off = block_off[blockIdx.x] + block_exclusive_scan(flag, total);
+    if (p <= n) cptr[p] = off;
+    if (flag) {
+        ckid[off] = kid_l[p];
+        cpos[off] = p;
+    }
+}
+
+// tab[(s * amax + l) * 2 + {0, 1}] = first compacted row of slot s in position l, and one past its last
+__global__ void position_table_kernel(const int32_t* __restrict__ slot_ptr, const int32_t* __restrict__ cptr, int n, int n_slots,
+                                      int amax, int32_t* __restrict__ tab) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_slots * amax) return;
+    const int s = i / amax, l = i % amax;
+    tab[2 * i] = cptr[(size_t)l * (n + 1) + slot_ptr[s]];
+    tab[2 * i + 1] = cptr[(size_t)l * (n + 1) + slot_ptr[s + 1]];
 }
 
 // Child-Sum cell, pointwise part, for the nodes at plan positions [lo, lo + m): Z rows (slot-local) hold W x + b
@@ -185,7 +221,7 @@ __global__ void childsum_pointwise_kernel(const int32_t* __restrict__ perm, cons
     }
 }
 
-// N-ary cell, pointwise part: G rows (slot-local, (3 + arity) H wide) hold sum_l U^l h_l (absent for a slot of leaves)
+// N-ary cell, pointwise part: G rows (by plan position, (3 + arity) H wide) hold sum_l U^l h_l (absent for a slot of leaves)
 __global__ void nary_pointwise_kernel(const int32_t* __restrict__ perm, const int32_t* __restrict__ kid, int n, int lo, int m, int H,
                                       int arity, const float* __restrict__ Z, const float* __restrict__ G, float* __restrict__ h,
                                       float* __restrict__ c, long long ldh) {
@@ -193,7 +229,7 @@ __global__ void nary_pointwise_kernel(const int32_t* __restrict__ perm, const in
     if (r >= m) return;
     const int j = perm[lo + r];
     const float* z = Z + (long long)r * 4 * H;
-    const float* g = G ? G + (long long)r * (3 + arity) * H : nullptr;
+    const float* g = G ? G + (long long)(lo + r) * (3 + arity) * H : nullptr;
     for (int col = threadIdx.x; col < H; col += blockDim.x) {
         const float i = sigmoidf_(z[col] + (g ? g[col] : 0.0f));
         const float o = sigmoidf_(z[H + col] + (g ? g[H + col] : 0.0f));
@@ -233,7 +269,7 @@ PlanWorkspace carve_plan(void* ws, long long n) {
 struct CellsWorkspace {
     float *Z, *G, *HS, *FE;
     int *edge_ptr, *slot_child, *slot_ppos, *block_sum, *flags;
-    int32_t *kid, *arity_of, *table;
+    int32_t *kid, *arity_of, *table, *cptr, *ckid, *cpos;
     size_t total;
 };
 CellsWorkspace carve_cells(void* ws, long long n, long long e, int H, int amax, int n_keys) {
@@ -251,7 +287,10 @@ CellsWorkspace carve_cells(void* ws, long long n, long long e, int H, int amax, 
     w.flags = (int*)take(4 * sizeof(int));
     w.kid = (int32_t*)take((size_t)(amax > 0 ? amax : 1) * n * sizeof(int32_t));
     w.arity_of = (int32_t*)take((size_t)(n_keys > 0 ? n_keys : 1) * sizeof(int32_t));
-    w.table = (int32_t*)take((size_t)3 * (n + 1) * sizeof(int32_t));
+    w.table = (int32_t*)take((size_t)2 * (amax > 0 ? amax : 1) * (n + 1) * sizeof(int32_t));
+    w.cptr = (int32_t*)take((size_t)(amax > 0 ? amax : 1) * (n + 1) * sizeof(int32_t));
+    w.ckid = (int32_t*)take((size_t)(amax > 0 ? amax : 1) * n * sizeof(int32_t));
+    w.cpos = (int32_t*)take((size_t)(amax > 0 ? amax : 1) * n * sizeof(int32_t));
     w.total = off;
     return w;
 }
@@ -357,8 +396,16 @@ jdb_status jdb_cells_forward(const jdb_forest* forest, const jdb_plan* plan, con
     slot_fill_kernel<<<sb, SCAN_BLOCK, 0, st>>>(forest->child_ptr, forest->child_idx, perm, n, ne, w.block_sum, w.edge_ptr, w.slot_child, w.slot_ppos);
     child_positions_kernel<<<ceil_div(n, 256), 256, 0, st>>>(forest->child_ptr, forest->child_idx, perm, key, w.arity_of, n, n_keys,
                                                            amax > 0 ? amax : 1, w.kid, w.flags);
+    for (int l = 1; l < amax; ++l) {   // position 0 is held by every internal node: no list needed
+        position_count_kernel<<<sb, SCAN_BLOCK, 0, st>>>(w.kid + (size_t)l * n, n, w.block_sum);
+        block_sums_scan_kernel<<<1, SCAN_BLOCK, 0, st>>>(w.block_sum, sb);
+        position_fill_kernel<<<sb, SCAN_BLOCK, 0, st>>>(w.kid + (size_t)l * n, n, w.block_sum, w.cptr + (size_t)l * (n + 1),
+                                                       w.ckid + (size_t)l * n, w.cpos + (size_t)l * n);
+    }
+    if (amax > 1) position_table_kernel<<<ceil_div((long long)S * amax, 256), 256, 0, st>>>(plan->slot_ptr, w.cptr, n, S, amax, w.table);
     JDB_CUDA_TRY(cudaGetLastError());
-    std::vector<int32_t> sp((size_t)S + 1), sd(S), sk(S), ep((size_t)n + 1);
+    std::vector<int32_t> sp((size_t)S + 1), sd(S), sk(S), ep((size_t)n + 1), tab(amax > 1 ? (size_t)2 * S * amax : 0);
+    if (amax > 1) JDB_CUDA_TRY(cudaMemcpyAsync(tab.data(), w.table, tab.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     int bad = 0;
     JDB_CUDA_TRY(cudaMemcpyAsync(sp.data(), plan->slot_ptr, sp.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     JDB_CUDA_TRY(cudaMemcpyAsync(sd.data(), plan->slot_depth, sd.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -380,7 +427,7 @@ jdb_status jdb_cells_forward(const jdb_forest* forest, const jdb_plan* plan, con
         {   // Z = x[rows] W^T + b
             GemmArgs g{};
             g.A = x; g.lda = ldx; g.a_idx = perm + lo; g.B = cl.W; g.ldb = D; g.C = w.Z; g.ldc = 4LL * H; g.M = m; g.N = 4 * H; g.K = D; g.bias = cl.b;
-            if ((r = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return r;
+            if ((r = gemm<true, false>(g, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
         }
         if (cl.kind == JDB_CELL_CHILDSUM) {
             const int e0 = ep[lo], e1 = ep[lo + m];
@@ -388,23 +435,30 @@ jdb_status jdb_cells_forward(const jdb_forest* forest, const jdb_plan* plan, con
                 child_sum_f32_kernel<<<ceil_div(m, pw_block.y), pw_block, 0, st>>>(forest->child_ptr, forest->child_idx, perm, lo, m, H, h, ldh, w.HS);
                 GemmArgs g{};
                 g.A = w.HS; g.lda = H; g.B = cl.U; g.ldb = H; g.C = w.Z; g.ldc = 4LL * H; g.M = m; g.N = 3 * H; g.K = H; g.beta = 1;
-                if ((r = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return r;
+                if ((r = gemm<true, false>(g, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
                 if (e1 > e0) {
                     GemmArgs f{};
                     f.A = h; f.lda = ldh; f.a_idx = w.slot_child + e0; f.B = cl.U + (size_t)3 * H * H; f.ldb = H; f.C = w.FE + (size_t)e0 * H; f.ldc = H;
                     f.M = e1 - e0; f.N = H; f.K = H;
-                    if ((r = gemm<true, false>(f, 0, n_sm, st)) != JDB_OK) return r;
+                    if ((r = gemm<true, false>(f, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
                 }
             }
             childsum_pointwise_kernel<<<ceil_div(m, pw_block.y), pw_block, 0, st>>>(perm, w.edge_ptr, w.slot_child, lo, m, H, w.Z, w.FE, h, c, ldh);
         } else {
             const int a = cl.arity;
             if (!leaves) {
-                for (int l = 0; l < a; ++l) {   // G (+)= h[child l] U^l T
+                const long long ldg = (3LL + a) * H;
+                for (int l = 0; l < a; ++l) {   // G (+)= h[child l] U^l T, over the rows that have a child l
                     GemmArgs g{};
-                    g.A = h; g.lda = ldh; g.a_idx = w.kid + (size_t)l * n + lo; g.B = cl.U + (size_t)l * H; g.ldb = (long long)a * H;
-                    g.C = w.G; g.ldc = (3LL + a) * H; g.M = m; g.N = (3 + a) * H; g.K = H; g.beta = l > 0;
-                    if ((r = gemm<true, false>(g, 0, n_sm, st)) != JDB_OK) return r;
+                    g.A = h; g.lda = ldh; g.B = cl.U + (size_t)l * H; g.ldb = (long long)a * H; g.ldc = ldg; g.N = (3 + a) * H; g.K = H;
+                    if (l == 0) {
+                        g.a_idx = w.kid + lo; g.C = w.G + (size_t)lo * ldg; g.M = m;
+                    } else {
+                        const int c0 = tab[((size_t)s * amax + l) * 2], c1 = tab[((size_t)s * amax + l) * 2 + 1];
+                        if (c1 <= c0) continue;
+                        g.a_idx = w.ckid + (size_t)l * n + c0; g.c_idx = w.cpos + (size_t)l * n + c0; g.C = w.G; g.M = c1 - c0; g.beta = 1;
+                    }
+                    if ((r = gemm<true, false>(g, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
                 }
             }
             nary_pointwise_kernel<<<ceil_div(m, pw_block.y), pw_block, 0, st>>>(perm, w.kid, n, lo, m, H, a, w.Z, leaves ? nullptr : w.G, h, c, ldh);
