@@ -343,6 +343,41 @@ jdb_status jdb_treelstm_forward_host(const int32_t *child_ptr, const int32_t *ch
                                      int32_t D, int32_t H, float *h, float *c, const jdb_opts *opts,
                                      void *dev_ws, size_t dev_ws_bytes, int32_t *n_levels_out, void *stream);
 
+/* ---- requests arriving one after the other (Section 2: serving, where requests arrive irregularly) ---------- */
+
+/* Every request is a forest of its own, given as HOST buffers (pinned memory makes the copies asynchronous).  A request
+ * takes the next of `slots` slots; a slot owns a stream and 1/slots of the caller's device scratch, so the copies and the
+ * batching analysis of a new request run while earlier requests execute, and nothing waits for a batch to fill.
+ * The object is host state only (streams, tickets); it allocates no device memory.  Not thread-safe: one thread submits
+ * and waits. */
+typedef struct jdb_online jdb_online;
+
+size_t jdb_online_workspace_bytes(int32_t slots, int32_t max_nodes, int32_t max_edges, int32_t D, int32_t H,
+                                  int32_t precision, int32_t x_dtype);
+
+/* slots 1 .. 16; max_nodes / max_edges bound a single request; packed from jdb_pack_weights (opts->precision, D, H);
+ * x_dtype of every request's x; dev_ws: jdb_online_workspace_bytes bytes of device memory, 256-byte aligned, owned by
+ * the caller and in use until jdb_online_destroy.  opts' timing events and trace are ignored. */
+jdb_status jdb_online_create(jdb_online **out, int32_t slots, int32_t max_nodes, int32_t max_edges, const void *packed,
+                             int32_t D, int32_t H, const jdb_opts *opts, int32_t x_dtype, void *dev_ws,
+                             size_t dev_ws_bytes);
+
+/* Enqueues one request (arguments as jdb_treelstm_forward_host: child_ptr, child_idx, x dense [n_nodes, D] in; h, c
+ * dense [n_nodes, H] out; all HOST pointers that must stay valid until the request has been waited for) and returns
+ * its ticket (0, 1, 2, ... in submission order).  If the slot it takes still holds an earlier request, that one is
+ * completed first (its status is kept for a later jdb_online_wait).  Does not wait for the new request, except that
+ * JDB_BF16 with H > 192 synchronises once for its level count.  A request larger than max_nodes / max_edges gives
+ * JDB_ERR_WORKSPACE and takes no ticket. */
+jdb_status jdb_online_submit(jdb_online *o, const int32_t *child_ptr, const int32_t *child_idx, int32_t n_nodes,
+                             int32_t n_edges, const void *x, float *h, float *c, int64_t *ticket);
+
+/* Waits for one request (in any order) and returns ITS status: JDB_OK, JDB_ERR_NOT_A_FOREST, JDB_ERR_TIMEOUT...; other
+ * requests are not affected by it.  n_levels_out (host, may be NULL) receives its level count. */
+jdb_status jdb_online_wait(jdb_online *o, int64_t ticket, int32_t *n_levels_out);
+
+/* Waits for everything in flight, destroys the streams and frees the host object. */
+jdb_status jdb_online_destroy(jdb_online *o);
+
 #ifdef __cplusplus
 }
 #endif

@@ -77,6 +77,79 @@ jdb_status schedule_common(const jdb_forest* f, jdb_sched* out, void* ws, size_t
 
 using namespace jdb;
 
+namespace jdb {
+// Copies a request's arrays to `dev_ws`, enqueues analysis, forward and the copies back on `stream`; does not wait for them
+// (except where the per-level launches need the level count: there the analysis synchronises).
+jdb_status forward_host_enqueue(const int32_t* child_ptr, const int32_t* child_idx, int32_t n_nodes, int32_t n_edges,
+                                const void* x, int32_t x_dtype, const void* packed, int32_t D, int32_t H, float* h, float* c,
+                                const jdb_opts* opts, void* dev_ws, size_t dev_ws_bytes, int32_t** meta_out, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_nodes < 0 || n_edges < 0 || !opts || D <= 0 || H <= 0) return JDB_ERR_INVALID_ARG;
+    if (x_dtype != JDB_FP32 && x_dtype != JDB_BF16) return JDB_ERR_INVALID_ARG;
+    *meta_out = nullptr;
+    if (n_nodes == 0) return n_edges == 0 ? JDB_OK : JDB_ERR_NOT_A_FOREST;
+    if (!child_ptr || (n_edges > 0 && !child_idx) || !x || !h || !c || !packed) return JDB_ERR_INVALID_ARG;
+    if (!dev_ws || ((uintptr_t)dev_ws & 255) != 0) return JDB_ERR_INVALID_ARG;
+    if (dev_ws_bytes < jdb_forward_host_workspace_bytes(n_nodes, n_edges, D, H, opts->precision, x_dtype))
+        return JDB_ERR_WORKSPACE;
+    const size_t n = (size_t)n_nodes, e = (size_t)(n_edges > 0 ? n_edges : 1), xb = x_dtype == JDB_BF16 ? 2 : 4;
+    char* p = (char*)dev_ws;
+    auto take = [&](size_t bytes) { char* q = p; p += align_up(bytes, 256); return q; };
+    int32_t* d_cp = (int32_t*)take((n + 1) * 4);
+    int32_t* d_ci = (int32_t*)take(e * 4);
+    void* d_x = take(n * (size_t)D * xb);
+    jdb_sched sch{};
+    sch.depth = (int32_t*)take(n * 4);
+    sch.perm = (int32_t*)take(n * 4);
+    sch.level_ptr = (int32_t*)take((n + 2) * 4);
+    sch.meta = (int32_t*)take(256);
+    const size_t ldh = ((size_t)H + 3) / 4 * 4;  // device rows padded to 16 bytes: the kernels' vector paths apply
+    float* d_h = (float*)take(n * ldh * 4);
+    float* d_c = (float*)take(n * ldh * 4);
+    size_t sws = schedule_ws_bytes(n_nodes, n_edges);
+    void* d_sws = take(sws);
+    size_t fws = jdb_forward_workspace_bytes(n_nodes, n_nodes, D, H, opts->precision);
+    void* d_fws = take(fws);
+
+    JDB_CUDA_TRY(cudaMemcpyAsync(d_cp, child_ptr, (n + 1) * 4, cudaMemcpyHostToDevice, st));
+    if (n_edges > 0) JDB_CUDA_TRY(cudaMemcpyAsync(d_ci, child_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice, st));
+    JDB_CUDA_TRY(cudaMemcpyAsync(d_x, x, n * (size_t)D * xb, cudaMemcpyHostToDevice, st));
+    jdb_forest f{d_cp, d_ci, n_nodes, n_edges};
+    // per-level launches (tensor-core path beyond the cooperative kernel's hidden sizes) need the level count on the
+    // host: there the analysis synchronises, and the forward is sized by the real number of internal nodes
+    const bool per_level = opts->precision == JDB_BF16 && !small_levels_supported(H);
+    jdb_status s = per_level ? jdb_schedule(&f, &sch, d_sws, sws, stream) : jdb_schedule_async(&f, &sch, d_sws, sws, stream);
+    if (s != JDB_OK) return s;
+    // enqueue the forward and the copies back before the one synchronisation
+    jdb_opts o = *opts;
+    o.mode = JDB_MODE_AUTO;
+    o.flags |= JDB_FLAG_NO_SYNC;  // the status is read once, together with the results
+    s = jdb_treelstm_forward(&f, &sch, d_x, x_dtype, D, packed, D, H, d_h, d_c, (int64_t)ldh, &o, d_fws, fws, stream);
+    if (s != JDB_OK) return s;
+    if (ldh == (size_t)H) {
+        JDB_CUDA_TRY(cudaMemcpyAsync(h, d_h, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
+        JDB_CUDA_TRY(cudaMemcpyAsync(c, d_c, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
+    } else {
+        JDB_CUDA_TRY(cudaMemcpy2DAsync(h, (size_t)H * 4, d_h, ldh * 4, (size_t)H * 4, n, cudaMemcpyDeviceToHost, st));
+        JDB_CUDA_TRY(cudaMemcpy2DAsync(c, (size_t)H * 4, d_c, ldh * 4, (size_t)H * 4, n, cudaMemcpyDeviceToHost, st));
+    }
+    *meta_out = sch.meta;
+    return JDB_OK;
+}
+
+// the status words of a request enqueued by forward_host_enqueue, after its stream has drained
+jdb_status forward_host_finish(const int32_t* meta_dev, int32_t* n_levels_out, void* stream) {
+    if (n_levels_out) *n_levels_out = 0;
+    if (!meta_dev) return JDB_OK;   // an empty forest: nothing was enqueued
+    int32_t meta[JDB_META_INTS];
+    jdb_status s = read_meta(meta_dev, meta, (cudaStream_t)stream);
+    if (s != JDB_OK) return s;
+    if (n_levels_out) *n_levels_out = meta[META_N_LEVELS];
+    return meta_status(meta);
+}
+
+}  // namespace jdb
+
 extern "C" {
 
 const char* jdb_status_string(jdb_status s) {
@@ -269,61 +342,12 @@ jdb_status jdb_treelstm_forward_host(const int32_t* child_ptr, const int32_t* ch
                                      int32_t n_edges, const void* x, int32_t x_dtype, const void* packed, int32_t D,
                                      int32_t H, float* h, float* c, const jdb_opts* opts, void* dev_ws,
                                      size_t dev_ws_bytes, int32_t* n_levels_out, void* stream) {
-    cudaStream_t st = (cudaStream_t)stream;
-    if (n_nodes < 0 || n_edges < 0 || !opts || D <= 0 || H <= 0) return JDB_ERR_INVALID_ARG;
-    if (x_dtype != JDB_FP32 && x_dtype != JDB_BF16) return JDB_ERR_INVALID_ARG;
     if (n_levels_out) *n_levels_out = 0;
-    if (n_nodes == 0) return n_edges == 0 ? JDB_OK : JDB_ERR_NOT_A_FOREST;
-    if (!child_ptr || (n_edges > 0 && !child_idx) || !x || !h || !c || !packed) return JDB_ERR_INVALID_ARG;
-    if (!dev_ws || ((uintptr_t)dev_ws & 255) != 0) return JDB_ERR_INVALID_ARG;
-    if (dev_ws_bytes < jdb_forward_host_workspace_bytes(n_nodes, n_edges, D, H, opts->precision, x_dtype))
-        return JDB_ERR_WORKSPACE;
-    const size_t n = (size_t)n_nodes, e = (size_t)(n_edges > 0 ? n_edges : 1), xb = x_dtype == JDB_BF16 ? 2 : 4;
-    char* p = (char*)dev_ws;
-    auto take = [&](size_t bytes) { char* q = p; p += align_up(bytes, 256); return q; };
-    int32_t* d_cp = (int32_t*)take((n + 1) * 4);
-    int32_t* d_ci = (int32_t*)take(e * 4);
-    void* d_x = take(n * (size_t)D * xb);
-    jdb_sched sch{};
-    sch.depth = (int32_t*)take(n * 4);
-    sch.perm = (int32_t*)take(n * 4);
-    sch.level_ptr = (int32_t*)take((n + 2) * 4);
-    sch.meta = (int32_t*)take(256);
-    const size_t ldh = ((size_t)H + 3) / 4 * 4;  // device rows padded to 16 bytes: the kernels' vector paths apply
-    float* d_h = (float*)take(n * ldh * 4);
-    float* d_c = (float*)take(n * ldh * 4);
-    size_t sws = schedule_ws_bytes(n_nodes, n_edges);
-    void* d_sws = take(sws);
-    size_t fws = jdb_forward_workspace_bytes(n_nodes, n_nodes, D, H, opts->precision);
-    void* d_fws = take(fws);
-
-    JDB_CUDA_TRY(cudaMemcpyAsync(d_cp, child_ptr, (n + 1) * 4, cudaMemcpyHostToDevice, st));
-    if (n_edges > 0) JDB_CUDA_TRY(cudaMemcpyAsync(d_ci, child_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice, st));
-    JDB_CUDA_TRY(cudaMemcpyAsync(d_x, x, n * (size_t)D * xb, cudaMemcpyHostToDevice, st));
-    jdb_forest f{d_cp, d_ci, n_nodes, n_edges};
-    // per-level launches (tensor-core path beyond the cooperative kernel's hidden sizes) need the level count on the
-    // host: there the analysis synchronises, and the forward is sized by the real number of internal nodes
-    const bool per_level = opts->precision == JDB_BF16 && !small_levels_supported(H);
-    jdb_status s = per_level ? jdb_schedule(&f, &sch, d_sws, sws, stream) : jdb_schedule_async(&f, &sch, d_sws, sws, stream);
+    int32_t* meta_dev = nullptr;
+    jdb_status s = forward_host_enqueue(child_ptr, child_idx, n_nodes, n_edges, x, x_dtype, packed, D, H, h, c, opts, dev_ws,
+                                        dev_ws_bytes, &meta_dev, stream);
     if (s != JDB_OK) return s;
-    // enqueue the forward and the copies back before the one synchronisation
-    jdb_opts o = *opts;
-    o.mode = JDB_MODE_AUTO;
-    o.flags |= JDB_FLAG_NO_SYNC;  // the status is read once, together with the results
-    s = jdb_treelstm_forward(&f, &sch, d_x, x_dtype, D, packed, D, H, d_h, d_c, (int64_t)ldh, &o, d_fws, fws, stream);
-    if (s != JDB_OK) return s;
-    if (ldh == (size_t)H) {
-        JDB_CUDA_TRY(cudaMemcpyAsync(h, d_h, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
-        JDB_CUDA_TRY(cudaMemcpyAsync(c, d_c, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
-    } else {
-        JDB_CUDA_TRY(cudaMemcpy2DAsync(h, (size_t)H * 4, d_h, ldh * 4, (size_t)H * 4, n, cudaMemcpyDeviceToHost, st));
-        JDB_CUDA_TRY(cudaMemcpy2DAsync(c, (size_t)H * 4, d_c, ldh * 4, (size_t)H * 4, n, cudaMemcpyDeviceToHost, st));
-    }
-    int32_t meta[JDB_META_INTS];
-    s = read_meta(sch.meta, meta, st);
-    if (s != JDB_OK) return s;
-    if (n_levels_out) *n_levels_out = meta[META_N_LEVELS];
-    return meta_status(meta);
+    return forward_host_finish(meta_dev, n_levels_out, stream);
 }
 
 }  // extern "C"

@@ -151,6 +151,14 @@ size_t forward_tc_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D,
 jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int n_levels, int n_internal_bound,
                               void* ws, bool use_small, uint64_t timeout_ns, cudaStream_t st);
 
+// ---- api.cu ----------------------------------------------------------------------------------
+// one request from host buffers: enqueue everything on `stream` (copies in, analysis, forward, copies back) without
+// waiting, and read the recorded status once the stream has drained
+jdb_status forward_host_enqueue(const int32_t* child_ptr, const int32_t* child_idx, int32_t n_nodes, int32_t n_edges,
+                                const void* x, int32_t x_dtype, const void* packed, int32_t D, int32_t H, float* h, float* c,
+                                const jdb_opts* opts, void* dev_ws, size_t dev_ws_bytes, int32_t** meta_out, void* stream);
+jdb_status forward_host_finish(const int32_t* meta_dev, int32_t* n_levels_out, void* stream);
+
 // ---- partition.cu -----------------------------------------------------------------------------
 // Tree partition for the cooperative level loop: nodes ordered by (depth, group) and the offsets of every
 // (depth, group) range; gbar holds one barrier counter per group (zeroed by partition_enqueue).

@@ -31,6 +31,7 @@ EXPORTS = [
     "jdb_treelstm_forward_host", "jdb_launch_counts_workspace_bytes", "jdb_launch_counts", "jdb_relatedness_head",
     "jdb_treelstm_backward_workspace_bytes", "jdb_treelstm_backward",
     "jdb_batch_plan_workspace_bytes", "jdb_batch_plan", "jdb_cells_forward_workspace_bytes", "jdb_cells_forward",
+    "jdb_online_workspace_bytes", "jdb_online_create", "jdb_online_submit", "jdb_online_wait", "jdb_online_destroy",
 ]
 CELL_CHILDSUM, CELL_NARY = 0, 1
 
@@ -117,6 +118,16 @@ def lib():
     L.jdb_cells_forward_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     L.jdb_cells_forward.restype = C.c_int
     L.jdb_cells_forward.argtypes = [vp, vp, vp, vp, i32, vp, i64, i32, i32, vp, vp, i64, vp, C.c_size_t, vp]
+    L.jdb_online_workspace_bytes.restype = C.c_size_t
+    L.jdb_online_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i32]
+    L.jdb_online_create.restype = C.c_int
+    L.jdb_online_create.argtypes = [vp, i32, i32, i32, vp, i32, i32, vp, i32, vp, C.c_size_t]
+    L.jdb_online_submit.restype = C.c_int
+    L.jdb_online_submit.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
+    L.jdb_online_wait.restype = C.c_int
+    L.jdb_online_wait.argtypes = [vp, i64, vp]
+    L.jdb_online_destroy.restype = C.c_int
+    L.jdb_online_destroy.argtypes = [vp]
     L.jdb_relatedness_head.restype = C.c_int
     L.jdb_relatedness_head.argtypes = [vp, i64, i32, vp, vp, i32, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.jdb_forward_host_workspace_bytes.restype = sz
@@ -488,3 +499,57 @@ def jdb_treelstm_forward_host(child_ptr: torch.Tensor, child_idx: torch.Tensor, 
     if st != OK:
         raise JdbError(st, "jdb_treelstm_forward_host")
     return nl.value
+
+
+class Online:
+    """Requests arriving one after the other: every request (a forest in host tensors) takes the next of `slots` slots, each
+    with its own stream and device scratch, so new requests are copied and analysed while earlier ones execute.
+
+    submit() returns a ticket; wait(ticket) returns that request's level count (its h and c host tensors are then
+    filled) or raises its error.  The host tensors of a request must stay alive until it has been waited for.
+    """
+
+    def __init__(self, slots: int, max_nodes: int, max_edges: int, packed: torch.Tensor, D: int, H: int, precision: int,
+                 x_dtype: int, device="cuda", flags: int = 0):
+        self.D, self.H, self.x_dtype = D, H, x_dtype
+        self.packed = packed
+        self.ws = _device_bytes(lib().jdb_online_workspace_bytes(slots, max_nodes, max_edges, D, H, precision, x_dtype), device)
+        opts = COpts(precision, MODE_AUTO, flags, 0, 0, None, None, None, None, 0)
+        self.handle = C.c_void_p(None)
+        st = lib().jdb_online_create(C.byref(self.handle), slots, max_nodes, max_edges, _ptr(packed), D, H, C.byref(opts), x_dtype,
+                                     _ptr(self.ws), self.ws.numel())
+        if st != OK:
+            raise JdbError(st, "jdb_online_create")
+        self._alive = {}
+
+    def submit(self, child_ptr: torch.Tensor, child_idx: torch.Tensor, x: torch.Tensor, h: torch.Tensor, c: torch.Tensor) -> int:
+        for t in (child_ptr, child_idx, x, h, c):
+            assert not t.is_cuda and t.is_contiguous()
+        assert (BF16 if x.dtype == torch.bfloat16 else FP32) == self.x_dtype
+        n, e = int(child_ptr.numel() - 1), int(child_idx.numel())
+        ticket = C.c_int64(-1)
+        st = lib().jdb_online_submit(self.handle, _ptr(child_ptr), _ptr(child_idx), n, e, _ptr(x), _ptr(h), _ptr(c), C.byref(ticket))
+        if st != OK:
+            raise JdbError(st, "jdb_online_submit")
+        self._alive[ticket.value] = (child_ptr, child_idx, x, h, c)
+        return ticket.value
+
+    def wait(self, ticket: int) -> int:
+        nl = C.c_int32(0)
+        st = lib().jdb_online_wait(self.handle, ticket, C.byref(nl))
+        self._alive.pop(ticket, None)
+        if st != OK:
+            raise JdbError(st, "jdb_online_wait")
+        return nl.value
+
+    def close(self):
+        if self.handle:
+            lib().jdb_online_destroy(self.handle)
+            self.handle = C.c_void_p(None)
+            self._alive.clear()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
