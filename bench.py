@@ -560,6 +560,60 @@ def time_batcher(idx: int, w: wl.Workload, device, flush, steps: int = 5, warmup
             "frac_of_fp32_alu_peak": flops / (tr * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS}
 
 
+def time_online(device, slots: int = 4, n_requests: int = 64, index: int = 2):
+    """A stream of requests (forests of workload 2's shape with 16 to 256 trees, pinned host buffers) through the
+    one-call host entry one after the other, and through jdb_online_* with `slots` requests in flight.  Host clock
+    around the whole stream, device idle on both sides.  Not part of `value`."""
+    import time
+    import torch
+    from paper_1904_07421_b200 import jdb
+    rng = np.random.default_rng(17)
+    base = wl.make_workload(index, n_trees=4)
+    precision = jdb.BF16 if base.precision == "bf16" else jdb.FP32
+    dt = torch.bfloat16 if precision == jdb.BF16 else torch.float32
+    packed = jdb.jdb_pack_weights(*(torch.from_numpy(a).to(device) for a in (base.W, base.U, base.b)), precision)
+    reqs = []
+    for k in range(n_requests):
+        wk = wl.make_workload(index, n_trees=int(rng.integers(16, 257)), seed=1000 + k)
+        f = wk.forest
+        x = torch.from_numpy(base.table[wk.token % base.table.shape[0]]).to(dt).pin_memory()
+        reqs.append((torch.from_numpy(f.child_ptr.astype(np.int32)).pin_memory(), torch.from_numpy(f.child_idx.astype(np.int32)).pin_memory(), x,
+                     torch.empty((f.n_nodes, wk.H), dtype=torch.float32).pin_memory(),
+                     torch.empty((f.n_nodes, wk.H), dtype=torch.float32).pin_memory(), f.n_nodes, f.n_trees, f.n_edges))
+    max_n, max_e = max(r[5] for r in reqs), max(r[7] for r in reqs)
+    ws = jdb.forward_host_workspace(max_n, max_e, base.D, base.H, precision, precision, device)
+    on = jdb.Online(slots, max_n, max_e, packed, base.D, base.H, precision, precision, device)
+
+    def serial():
+        for r in reqs:
+            jdb.jdb_treelstm_forward_host(r[0], r[1], r[2], packed, base.D, base.H, precision, r[3], r[4], ws)
+
+    def online():
+        tickets = [on.submit(*r[:5]) for r in reqs]
+        for t in tickets:
+            on.wait(t)
+
+    out = {}
+    for name, fn_ in (("one_call_entries", serial), ("online", online)):
+        fn_()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(5):
+            t0 = time.perf_counter()
+            fn_()
+            torch.cuda.synchronize()
+            ts.append(time.perf_counter() - t0)
+        out[name] = statistics.median(ts)
+    on.close()
+    nodes, trees = sum(r[5] for r in reqs), sum(r[6] for r in reqs)
+    return {"workload": f"{n_requests} requests of workload {index}'s shape, 16-256 trees each ({trees} trees, {nodes} nodes), "
+                        "pinned host buffers in and out", "slots": slots,
+            "one_call_entries": {"seconds": out["one_call_entries"], "requests_per_s": n_requests / out["one_call_entries"],
+                                 "nodes_per_s": nodes / out["one_call_entries"]},
+            "online": {"seconds": out["online"], "requests_per_s": n_requests / out["online"], "nodes_per_s": nodes / out["online"]},
+            "speedup": out["one_call_entries"] / out["online"]}
+
+
 def rank_workload(config: int, rank: int, n_trees=None) -> wl.Workload:
     """Every rank draws its own forest of the workload's shape (weak scaling over independent trees)."""
     return wl.make_workload(config, n_trees=n_trees, seed=None if rank == 0 else wl.BASE_SEED + config + 1000 * rank)
@@ -620,7 +674,8 @@ def run_gpu(args):
         flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=device)
         wt = wl.make_workload(args.training_only, n_trees=args.trees)
         print(json.dumps({"training": [time_training(args.training_only, wt, device, flush, args.steps, args.warmup)],
-                          "keyed_batcher": [time_batcher(args.training_only, wt, device, flush, args.steps, args.warmup)]}))
+                          "keyed_batcher": [time_batcher(args.training_only, wt, device, flush, args.steps, args.warmup)],
+                          "online_requests": time_online(device) if args.training_only == 2 else None}))
         return
     pk = peaks()
     mode = {"auto": jdb.MODE_AUTO, "level": jdb.MODE_PER_LEVEL, "persistent": jdb.MODE_PERSISTENT}[args.mode]
@@ -686,6 +741,7 @@ def run_gpu(args):
                 if b is not None:
                     batcher.append(b)
                 torch.cuda.empty_cache()
+        online = time_online(device) if (args.all_configs and world == 1) else None
         cpu_v, cpu_sample, cpu_trees = time_oracle(w, args.cpu_budget)
         cpu_par = None
         if args.cpu_budget >= 1.0:
@@ -711,6 +767,7 @@ def run_gpu(args):
             "relatedness_head": head,
             "training": training,
             "keyed_batcher": batcher,
+            "online_requests": online,
             "batching_ratio": f.n_nodes / max(n_levels_main, 1),   # cells evaluated per batched step: Section 3's batching ratio at cell granularity
             "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_sample,
                              "parallel_over_trees": cpu_par},
