@@ -149,6 +149,33 @@ def test_gradient_of_some_trees_equals_the_subforest():
     assert np.all(dx[others] == 0.0)
 
 
+def test_large_forest_sampled_trees():
+    """Workload 5's shape at 12288 trees (about 290 k nodes, D = H = 1024): the gradient rows of the workspace pass the
+    2^31 and 2^32 byte offsets, the edge-slot scan spans several hundred blocks, the parameter gradients split their
+    contraction many ways.  Loss on a sample of trees (the first, the last, the owners of the rows at those offsets and
+    random ones); the checker runs on their sub-forest (about 10 s)."""
+    w = dataclasses.replace(wl.make_workload(5, n_trees=12288, bias="random"), precision="fp32")
+    f = w.forest
+    rng = np.random.default_rng(29)
+    rows = [0, f.n_nodes - 1] + [(1 << s) // (4 * 4 * w.H) + k for s in (31, 32) for k in (-1, 0, 1)]
+    trees = np.unique(np.concatenate([np.searchsorted(f.tree_ptr, np.asarray(rows), side="right") - 1,
+                                      rng.choice(f.n_trees, size=6, replace=False)]))
+    sub, nodes = wl.subforest(f, trees)
+    gh = np.zeros((f.n_nodes, w.H), dtype=np.float32)
+    gc = np.zeros((f.n_nodes, w.H), dtype=np.float32)
+    gh[nodes] = rng.standard_normal((len(nodes), w.H))
+    gc[nodes] = rng.standard_normal((len(nodes), w.H)) * 0.5
+    dW, dU, db, dx = _run(w, gh, gc)
+    ref = ob.backward(sub.child_ptr, sub.child_idx, w.x_rows(nodes), w.W, w.U, w.b, gh[nodes], gc[nodes])
+    _close(dW, ref[0], "dW")
+    _close(dU, ref[1], "dU")
+    _close(db, ref[2], "db")
+    _close(dx[nodes], ref[3], "dx")
+    mask = np.ones(f.n_nodes, dtype=bool)
+    mask[nodes] = False
+    assert not dx[mask].any()
+
+
 def test_empty_forest_and_argument_errors():
     dev = torch.device("cuda:0")
     a = wl.make_custom([[-1, 0, 0, 1]], D=4, H=4, seed=1)

@@ -41,6 +41,14 @@ def test_table_is_bit_exact(index, n_trees, n_keys):
     _check_plan(f, rng.integers(0, n_keys, size=f.n_nodes), n_keys)
 
 
+def test_table_at_full_size():
+    """Workload 5's whole forest (1.57 M nodes): 1535 scan blocks (the scanning CTA walks its block sums in two rounds)
+    and 768 sort tiles."""
+    rng = np.random.default_rng(77)
+    f = wl.make_forest(5, rng)
+    _check_plan(f, rng.integers(0, 3, size=f.n_nodes), 3)
+
+
 def test_table_edge_cases():
     one = wl.forest_from_parents([np.asarray([-1])])
     _check_plan(one, [0], 1)
