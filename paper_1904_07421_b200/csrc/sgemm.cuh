@@ -89,8 +89,8 @@ __device__ __forceinline__ void store_tile(float (*S)[LDS_], int t, const float 
 // B(k, n) = B[row(k) * ldb + n] (B_ROW_K) or B[n * ldb + k].
 template <bool A_ROW_M, bool B_ROW_K>
 __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
-    __shared__ __align__(16) float As[BK][LDS_];
-    __shared__ __align__(16) float Bs[BK][LDS_];
+    __shared__ __align__(16) float As[2][BK][LDS_];   // two buffers: the next tile is stored while this one is read,
+    __shared__ __align__(16) float Bs[2][BK][LDS_];   // one barrier per K step
     const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
     // tiles that share rows of A are neighbours in the grid: A reaches DRAM once, B (the smaller operand) stays in L2
     const int m0 = (blockIdx.x / g.tn) * BM, n0 = (blockIdx.x % g.tn) * BN;
@@ -106,21 +106,23 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
     if (kbeg < kend) {
         load_tile<A_ROW_M>(g.A, g.lda, g.a_idx, m0, g.M, kbeg, kend, g.vec_a, t, ra);
         load_tile<!B_ROW_K>(g.B, g.ldb, g.b_idx, n0, g.N, kbeg, kend, g.vec_b, t, rb);
+        store_tile<A_ROW_M>(As[0], t, ra);
+        store_tile<!B_ROW_K>(Bs[0], t, rb);
     }
+    __syncthreads();
+    int cur = 0;
     for (int k0 = kbeg; k0 < kend; k0 += BK) {
-        store_tile<A_ROW_M>(As, t, ra);
-        store_tile<!B_ROW_K>(Bs, t, rb);
-        __syncthreads();
-        if (k0 + BK < kend) {   // the next tile's loads fly while this one is multiplied
+        const bool more = k0 + BK < kend;
+        if (more) {   // the next tile's loads fly while this one is multiplied
             load_tile<A_ROW_M>(g.A, g.lda, g.a_idx, m0, g.M, k0 + BK, kend, g.vec_a, t, ra);
             load_tile<!B_ROW_K>(g.B, g.ldb, g.b_idx, n0, g.N, k0 + BK, kend, g.vec_b, t, rb);
         }
 #pragma unroll
         for (int k = 0; k < BK; ++k) {
-            const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[k][64 + ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
-            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[k][64 + tx * 4]);
+            const float4 a0 = *reinterpret_cast<const float4*>(&As[cur][k][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4*>(&As[cur][k][64 + ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[cur][k][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[cur][k][64 + tx * 4]);
             const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
             const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
@@ -128,7 +130,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2) sgemm_kernel(GemmArgs g) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
+        if (more) {   // the other buffer was last read one step ago, before the barrier that ended that step
+            store_tile<A_ROW_M>(As[cur ^ 1], t, ra);
+            store_tile<!B_ROW_K>(Bs[cur ^ 1], t, rb);
+        }
         __syncthreads();
+        cur ^= 1;
     }
     if (kbeg >= kend && blockIdx.z > 0) return;
 
