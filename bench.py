@@ -433,6 +433,47 @@ def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device
     return ms, h2d, d2h
 
 
+def time_e2e_pipelined(w: wl.Workload, job_precision, packed, steps: int, warmup: int, flush, device, chunks: int = 8, slots: int = 3):
+    """The same end-to-end step with the forest handed over in `chunks` groups of whole trees through jdb_online_*: the
+    copies in of one group, the execution of another and the copies back of a third overlap.  Returns per-step ms."""
+    import torch
+    from paper_1904_07421_b200 import jdb
+    f = w.forest
+    dt = torch.bfloat16 if job_precision == jdb.BF16 else torch.float32
+    bounds = np.linspace(0, f.n_trees, min(chunks, f.n_trees) + 1).astype(np.int64)
+    parts = []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        sub, nodes = wl.subforest(f, np.arange(a, b))
+        parts.append((torch.from_numpy(sub.child_ptr.astype(np.int32)).pin_memory(), torch.from_numpy(sub.child_idx.astype(np.int32)).pin_memory(),
+                      torch.from_numpy(w.x_rows(nodes)).to(dt).pin_memory(),
+                      torch.empty((len(nodes), w.H), dtype=torch.float32).pin_memory(),
+                      torch.empty((len(nodes), w.H), dtype=torch.float32).pin_memory(), sub.n_edges))
+    on = jdb.Online(slots, max(p[3].shape[0] for p in parts), max(p[5] for p in parts), packed, w.D, w.H, job_precision,
+                    jdb.BF16 if dt == torch.bfloat16 else jdb.FP32, device)
+
+    def step():
+        tickets = [on.submit(*p[:5]) for p in parts]
+        for t in tickets:
+            on.wait(t)
+
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(steps):
+        flush.add_(1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        torch.cuda.synchronize()
+        e1.record()
+        e1.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    on.close()
+    return ms
+
+
 def time_head(w: wl.Workload, job: GpuJob, flush, pk, Hs: int = 50, K: int = 5, reps: int = 10):
     """The relatedness head over the forest's root states (pairs of consecutive trees): time per call and the
     fraction of the copy bandwidth its algorithmic bytes (two root rows per pair) reach.  Not part of `value`."""
@@ -714,6 +755,10 @@ def run_gpu(args):
     e2e_ms, h2d, d2h = time_e2e(w, job, args.steps, args.warmup, flush, device)
     t_e2e_s, _ = job_totals(sum(e2e_ms) / 1e3, f.n_nodes, world, device)
     e2e_value = total_nodes * args.steps / t_e2e_s
+    torch.cuda.empty_cache()
+    pipe_ms = time_e2e_pipelined(w, precision_main, packed_main, args.steps, args.warmup, flush, device)
+    t_pipe_s, _ = job_totals(sum(pipe_ms) / 1e3, f.n_nodes, world, device)
+    pipe_value = total_nodes * args.steps / t_pipe_s
     del job
     torch.cuda.empty_cache()
 
@@ -758,8 +803,13 @@ def run_gpu(args):
                        **({"reduced_to_trees": args.trees} if args.trees else {}),
                        "l2": "256 MiB buffer rewritten between timed steps", "parallelism": f"tree-sharded x{world}"},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": 1e3 * t_e2e_s / args.steps},
+            # the better of the two ways a caller has: one call for the whole forest, or the forest handed over in eight
+            # groups of whole trees through jdb_online_* (three slots), whose copies and execution overlap
+            "e2e": {"value": max(e2e_value, pipe_value), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": 1e3 * min(t_e2e_s, t_pipe_s) / args.steps,
+                    "entry": "jdb_online_* (8 groups of trees, 3 slots)" if pipe_value > e2e_value else "jdb_treelstm_forward_host",
+                    "one_call": {"value": e2e_value, "ms_per_step": 1e3 * t_e2e_s / args.steps},
+                    "pipelined": {"value": pipe_value, "ms_per_step": 1e3 * t_pipe_s / args.steps}},
             "gpu_launches": launches_main * args.steps,
             "roofline": roofline,
             "path_frac_of_roofline": path_frac,

@@ -113,13 +113,14 @@ jdb_status forward_host_enqueue(const int32_t* child_ptr, const int32_t* child_i
 
     JDB_CUDA_TRY(cudaMemcpyAsync(d_cp, child_ptr, (n + 1) * 4, cudaMemcpyHostToDevice, st));
     if (n_edges > 0) JDB_CUDA_TRY(cudaMemcpyAsync(d_ci, child_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice, st));
-    JDB_CUDA_TRY(cudaMemcpyAsync(d_x, x, n * (size_t)D * xb, cudaMemcpyHostToDevice, st));
     jdb_forest f{d_cp, d_ci, n_nodes, n_edges};
     // per-level launches (tensor-core path beyond the cooperative kernel's hidden sizes) need the level count on the
-    // host: there the analysis synchronises, and the forward is sized by the real number of internal nodes
+    // host: there the analysis synchronises, and the forward is sized by the real number of internal nodes.  The copy
+    // of x follows the analysis, so that this wait covers the CSR and the analysis only.
     const bool per_level = opts->precision == JDB_BF16 && !small_levels_supported(H);
     jdb_status s = per_level ? jdb_schedule(&f, &sch, d_sws, sws, stream) : jdb_schedule_async(&f, &sch, d_sws, sws, stream);
     if (s != JDB_OK) return s;
+    JDB_CUDA_TRY(cudaMemcpyAsync(d_x, x, n * (size_t)D * xb, cudaMemcpyHostToDevice, st));
     // enqueue the forward and the copies back before the one synchronisation
     jdb_opts o = *opts;
     o.mode = JDB_MODE_AUTO;
