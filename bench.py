@@ -403,7 +403,7 @@ def time_steps(job: GpuJob, steps: int, warmup: int, flush, timed_events=False):
     return total, level_ms
 
 
-def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device):
+def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device, roots_only: bool = False):
     """The same step through the host-buffer entry point: pinned host arrays in, pinned host arrays out, the
     copies inside the timed region.  Returns (per-step ms, h2d bytes, d2h bytes)."""
     torch, jdb = job.torch, job.jdb
@@ -411,12 +411,14 @@ def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device
     dt = torch.bfloat16 if job.precision == jdb.BF16 else torch.float32
     hx = torch.from_numpy(w.x_full()).to(dt).pin_memory()
     hcp, hci = torch.from_numpy(f.child_ptr).pin_memory(), torch.from_numpy(f.child_idx).pin_memory()
-    hh = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
-    hc = torch.empty((f.n_nodes, w.H), dtype=torch.float32).pin_memory()
+    rows = f.n_nodes - f.n_edges if roots_only else f.n_nodes   # with JDB_FLAG_ROOTS_ONLY only the roots' states come back
+    flags = jdb.FLAG_ROOTS_ONLY if roots_only else 0
+    hh = torch.empty((rows, w.H), dtype=torch.float32).pin_memory()
+    hc = torch.empty((rows, w.H), dtype=torch.float32).pin_memory()
     x_dtype = jdb.BF16 if dt == torch.bfloat16 else jdb.FP32
     hws = jdb.forward_host_workspace(f.n_nodes, f.n_edges, w.D, w.H, job.precision, x_dtype, device)
     for _ in range(max(warmup, 3)):
-        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
+        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws, flags=flags)
     torch.cuda.synchronize()
     ms = []
     for _ in range(steps):
@@ -424,7 +426,7 @@ def time_e2e(w: wl.Workload, job: GpuJob, steps: int, warmup: int, flush, device
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws)
+        jdb.jdb_treelstm_forward_host(hcp, hci, hx, job.packed, w.D, w.H, job.precision, hh, hc, hws, flags=flags)
         e1.record()
         e1.synchronize()
         ms.append(e0.elapsed_time(e1))
@@ -756,6 +758,9 @@ def run_gpu(args):
     t_e2e_s, _ = job_totals(sum(e2e_ms) / 1e3, f.n_nodes, world, device)
     e2e_value = total_nodes * args.steps / t_e2e_s
     torch.cuda.empty_cache()
+    roots_ms, _, roots_d2h = time_e2e(w, job, args.steps, args.warmup, flush, device, roots_only=True)
+    t_roots_s, _ = job_totals(sum(roots_ms) / 1e3, f.n_nodes, world, device)
+    torch.cuda.empty_cache()
     pipe_ms = time_e2e_pipelined(w, precision_main, packed_main, args.steps, args.warmup, flush, device)
     t_pipe_s, _ = job_totals(sum(pipe_ms) / 1e3, f.n_nodes, world, device)
     pipe_value = total_nodes * args.steps / t_pipe_s
@@ -809,7 +814,11 @@ def run_gpu(args):
                     "ms_per_step": 1e3 * min(t_e2e_s, t_pipe_s) / args.steps,
                     "entry": "jdb_online_* (8 groups of trees, 3 slots)" if pipe_value > e2e_value else "jdb_treelstm_forward_host",
                     "one_call": {"value": e2e_value, "ms_per_step": 1e3 * t_e2e_s / args.steps},
-                    "pipelined": {"value": pipe_value, "ms_per_step": 1e3 * t_pipe_s / args.steps}},
+                    "pipelined": {"value": pipe_value, "ms_per_step": 1e3 * t_pipe_s / args.steps},
+                    # the one call with JDB_FLAG_ROOTS_ONLY: only the roots' states cross back (what a sentence-level
+                    # task reads); not the line's e2e value, which returns every node's state
+                    "roots_only": {"value": total_nodes * args.steps / t_roots_s, "ms_per_step": 1e3 * t_roots_s / args.steps,
+                                   "d2h_bytes_per_step": roots_d2h}},
             "gpu_launches": launches_main * args.steps,
             "roofline": roofline,
             "path_frac_of_roofline": path_frac,

@@ -48,6 +48,9 @@ enum { JDB_MODE_AUTO = 0, JDB_MODE_PER_LEVEL = 1, JDB_MODE_PERSISTENT = 2 };
 /* jdb_opts.flags */
 enum {
     JDB_FLAG_NO_SYNC = 1,      /* jdb_treelstm_forward never synchronises; ask jdb_sched_status afterwards */
+    JDB_FLAG_ROOTS_ONLY = 4,   /* host entries (jdb_treelstm_forward_host, jdb_online_submit) only: h and c receive the
+                                  states of the ROOTS alone, dense [n_nodes - n_edges, H], roots in ascending node id
+                                  (what a sentence-level task reads; the other rows stay on the device)            */
     JDB_FLAG_DEBUG_CHECKS = 2  /* every kernel of the forward pass checks the indices it is about to follow (child ids,
                                   positions in level order, level offsets, rows of the workspace arrays) against the
                                   sizes of the arrays they index, skips an access that would leave them and records the

@@ -2,6 +2,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "scan.cuh"
 
 namespace jdb {
 static thread_local int g_last_cuda_error = 0;
@@ -25,6 +26,38 @@ DevInfo* dev_info() {
 }
 
 namespace {
+
+// ---- roots only: the rows of the nodes that no child list mentions, compacted in ascending id ----------------------
+__global__ void mark_children_kernel(const int32_t* __restrict__ child_idx, int n_edges, int n, int* __restrict__ is_child) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n_edges) return;
+    const int c = child_idx[e];
+    if (c >= 0 && c < n) is_child[c] = 1;
+}
+__global__ void __launch_bounds__(SCAN_BLOCK) root_count_kernel(const int* __restrict__ is_child, int n, int* block_sum) {
+    const int v = blockIdx.x * SCAN_BLOCK + threadIdx.x;
+    int total;
+    block_exclusive_scan((v < n && !is_child[v]) ? 1 : 0, total);
+    if (threadIdx.x == 0) block_sum[blockIdx.x] = total;
+}
+__global__ void __launch_bounds__(SCAN_BLOCK) root_list_kernel(const int* __restrict__ is_child, int n, const int* block_off, int n_roots,
+                                                               int32_t* __restrict__ root_id) {
+    const int v = blockIdx.x * SCAN_BLOCK + threadIdx.x;
+    const int flag = (v < n && !is_child[v]) ? 1 : 0;
+    int total;
+    const int r = block_off[blockIdx.x] + block_exclusive_scan(flag, total);
+    if (flag && r < n_roots) root_id[r] = v;
+}
+__global__ void root_rows_kernel(const int32_t* __restrict__ root_id, int n_roots, int H, const float* __restrict__ h,
+                                 const float* __restrict__ c, long long ldh, float* __restrict__ hr, float* __restrict__ cr) {
+    const int r = blockIdx.x * blockDim.y + threadIdx.y;
+    if (r >= n_roots) return;
+    const long long v = root_id[r];
+    for (int col = threadIdx.x; col < H; col += blockDim.x) {
+        hr[(long long)r * H + col] = h[v * ldh + col];
+        cr[(long long)r * H + col] = c[v * ldh + col];
+    }
+}
 
 jdb_status read_meta(const int32_t* meta_dev, int32_t* meta_host, cudaStream_t st) {
     JDB_CUDA_TRY(cudaMemcpyAsync(meta_host, meta_dev, JDB_META_INTS * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -124,10 +157,31 @@ jdb_status forward_host_enqueue(const int32_t* child_ptr, const int32_t* child_i
     // enqueue the forward and the copies back before the one synchronisation
     jdb_opts o = *opts;
     o.mode = JDB_MODE_AUTO;
-    o.flags |= JDB_FLAG_NO_SYNC;  // the status is read once, together with the results
+    o.flags = (o.flags | JDB_FLAG_NO_SYNC) & ~JDB_FLAG_ROOTS_ONLY;  // the status is read once, together with the results
     s = jdb_treelstm_forward(&f, &sch, d_x, x_dtype, D, packed, D, H, d_h, d_c, (int64_t)ldh, &o, d_fws, fws, stream);
     if (s != JDB_OK) return s;
-    if (ldh == (size_t)H) {
+    if (opts->flags & JDB_FLAG_ROOTS_ONLY) {
+        int* is_child = (int*)take(n * 4);
+        int32_t* root_id = (int32_t*)take(n * 4);
+        int* block_sum = (int*)take((n / SCAN_BLOCK + 2) * 4);
+        float* hr = (float*)take(n * (size_t)H * 4);
+        float* cr = (float*)take(n * (size_t)H * 4);
+        const int n_roots = n_nodes > n_edges ? n_nodes - n_edges : 0;   // every other node has exactly one parent edge
+        const int sb = n_nodes / SCAN_BLOCK + 1;
+        JDB_CUDA_TRY(cudaMemsetAsync(is_child, 0, n * 4, st));
+        if (n_edges > 0) mark_children_kernel<<<ceil_div(n_edges, 256), 256, 0, st>>>(d_ci, n_edges, n_nodes, is_child);
+        root_count_kernel<<<sb, SCAN_BLOCK, 0, st>>>(is_child, n_nodes, block_sum);
+        block_sums_scan_kernel<<<1, SCAN_BLOCK, 0, st>>>(block_sum, sb);
+        root_list_kernel<<<sb, SCAN_BLOCK, 0, st>>>(is_child, n_nodes, block_sum, n_roots, root_id);
+        if (n_roots > 0) {
+            const dim3 blk(H >= 128 ? 128 : 32, H >= 128 ? 2 : 8);
+            root_rows_kernel<<<ceil_div(n_roots, blk.y), blk, 0, st>>>(root_id, n_roots, H, d_h, d_c, (long long)ldh, hr, cr);
+            JDB_CUDA_TRY(cudaGetLastError());
+            JDB_CUDA_TRY(cudaMemcpyAsync(h, hr, (size_t)n_roots * H * 4, cudaMemcpyDeviceToHost, st));
+            JDB_CUDA_TRY(cudaMemcpyAsync(c, cr, (size_t)n_roots * H * 4, cudaMemcpyDeviceToHost, st));
+        }
+        JDB_CUDA_TRY(cudaGetLastError());
+    } else if (ldh == (size_t)H) {
         JDB_CUDA_TRY(cudaMemcpyAsync(h, d_h, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
         JDB_CUDA_TRY(cudaMemcpyAsync(c, d_c, n * (size_t)H * 4, cudaMemcpyDeviceToHost, st));
     } else {
@@ -336,6 +390,8 @@ size_t jdb_forward_host_workspace_bytes(int32_t n_nodes, int32_t n_edges, int32_
     bytes += 2 * align_up(n * (((size_t)H + 3) / 4 * 4) * 4, 256);         // h, c (rows padded to 16 bytes)
     bytes += align_up(schedule_ws_bytes(n_nodes, n_edges), 256);
     bytes += jdb_forward_workspace_bytes(n_nodes, n_nodes, D, H, precision);
+    // JDB_FLAG_ROOTS_ONLY: child marks, root ids, block sums, and the compacted rows (at most every node is a root)
+    bytes += 2 * align_up(n * 4, 256) + align_up((n / SCAN_BLOCK + 2) * 4, 256) + 2 * align_up(n * (size_t)H * 4, 256);
     return bytes;
 }
 

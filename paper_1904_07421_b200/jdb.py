@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libjdb.so")
 
 OK, ERR_INVALID_ARG, ERR_NOT_A_FOREST, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_CHECK = range(8)
 FP32, BF16 = 0, 1
-FLAG_NO_SYNC, FLAG_DEBUG_CHECKS = 1, 2
+FLAG_NO_SYNC, FLAG_DEBUG_CHECKS, FLAG_ROOTS_ONLY = 1, 2, 4
 TUNE_SET, TUNE_PAIR_XPROJ, TUNE_PAIR_LEVEL, TUNE_PAIR_FORGET, TUNE_TWO_ISSUERS, TUNE_NO_PDL, TUNE_PLAIN_STORES = 1, 2, 4, 8, 16, 32, 64
 TUNE_GATHER_X, TUNE_TREE_GROUPS = 128, 256
 MODE_AUTO, MODE_PER_LEVEL, MODE_PERSISTENT = 0, 1, 2

@@ -105,3 +105,32 @@ def test_an_error_stays_with_its_request_and_limits_are_enforced():
                   torch.zeros((0, base.H)), torch.zeros((0, base.H)))
     assert on.wait(e) == 0
     on.close()
+
+
+@pytest.mark.parametrize("index,n_trees", [(1, 50), (2, 120), (3, 20)])
+def test_roots_only_returns_the_root_rows(index, n_trees):
+    """JDB_FLAG_ROOTS_ONLY: the host entries hand back the states of the roots alone, ascending by node id, bit for bit
+    the rows of the full result (fp32, bf16 cooperative loop, bf16 per-level launches; ids shuffled so that roots are
+    scattered over the id range)."""
+    w0 = wl.make_workload(index, n_trees=n_trees, bias="random")
+    forest, new_of_old = wl.relabel(w0.forest, np.random.default_rng(3))
+    token = np.empty_like(w0.token)
+    token[new_of_old] = w0.token
+    w = wl.Workload(w0.name, w0.index, forest, w0.D, w0.H, w0.precision, w0.table, token, w0.W, w0.U, w0.b)
+    f = w.forest
+    precision = jdb.BF16 if w.precision == "bf16" else jdb.FP32
+    packed = jdb.jdb_pack_weights(*(torch.from_numpy(a).to(DEV) for a in (w.W, w.U, w.b)), precision)
+    cp, ci, x, h, c = _request(w)
+    ws = jdb.forward_host_workspace(f.n_nodes, f.n_edges, w.D, w.H, precision, precision, DEV)
+    jdb.jdb_treelstm_forward_host(cp, ci, x, packed, w.D, w.H, precision, h, c, ws)
+    roots = np.sort(np.asarray(f.roots, dtype=np.int64))
+    assert len(roots) == f.n_nodes - f.n_edges
+    hr = torch.full((len(roots), w.H), float("nan")).pin_memory()
+    cr = torch.full((len(roots), w.H), float("nan")).pin_memory()
+    jdb.jdb_treelstm_forward_host(cp, ci, x, packed, w.D, w.H, precision, hr, cr, ws, flags=jdb.FLAG_ROOTS_ONLY)
+    assert torch.equal(hr, h[roots]) and torch.equal(cr, c[roots])
+    on = jdb.Online(2, f.n_nodes, f.n_edges, packed, w.D, w.H, precision, precision, DEV, flags=jdb.FLAG_ROOTS_ONLY)
+    hr2, cr2 = torch.full_like(hr, float("nan")).pin_memory(), torch.full_like(cr, float("nan")).pin_memory()
+    on.wait(on.submit(cp, ci, x, hr2, cr2))
+    on.close()
+    assert torch.equal(hr2, hr) and torch.equal(cr2, cr)
