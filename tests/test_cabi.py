@@ -41,6 +41,20 @@ def test_host_only_queries():
     assert fw >= 400 * 600 * 4
     hw = L.jdb_forward_host_workspace_bytes(1000, 999, 300, 150, jdb.FP32, jdb.FP32)
     assert hw > fw + 2 * 1000 * 150 * 4
+    # the entry points added beside the forward: sizes grow with what they hold, bad sizes give 0
+    bw = L.jdb_treelstm_backward_workspace_bytes(1000, 999, 400, 150)
+    assert bw >= (1000 * 4 * 150 + 2 * 1000 * 150 + 999 * 150) * 4 and L.jdb_treelstm_backward_workspace_bytes(-1, 0, 0, 150) == 0
+    assert L.jdb_batch_plan_workspace_bytes(100000) >= 3 * 100000 * 4
+    cw2, cw8 = (L.jdb_cells_forward_workspace_bytes(1000, 999, 150, a, 2) for a in (2, 8))
+    assert 1000 * 4 * 150 * 4 < cw2 < cw8
+    assert L.jdb_online_workspace_bytes(3, 1000, 999, 300, 150, jdb.FP32, jdb.FP32) >= 3 * hw
+    assert L.jdb_online_workspace_bytes(0, 1000, 999, 300, 150, jdb.FP32, jdb.FP32) == 0
+    # the host object of the online entry refuses bad arguments before it touches the device
+    handle = ctypes.c_void_p(None)
+    opts = jdb.COpts(jdb.FP32, jdb.MODE_AUTO, 0, 0, 0, None, None, None, None, 0)
+    assert L.jdb_online_create(ctypes.byref(handle), 0, 10, 9, None, 4, 4, ctypes.byref(opts), jdb.FP32, None, 0) == jdb.ERR_INVALID_ARG
+    assert not handle.value
+    assert L.jdb_online_destroy(None) == jdb.OK
 
 
 def L_places(n):
@@ -53,4 +67,6 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(jdb.CSched) == 48
     assert ctypes.sizeof(jdb.COpts) == 64
     assert ctypes.sizeof(jdb.CLaunchStats) == 40
+    assert ctypes.sizeof(jdb.CPlan) == 40       # four pointers, two int32
+    assert ctypes.sizeof(jdb.CCell) == 32       # two int32, three pointers
     assert L_places(1) >= 1024 * 8 and L_places(100000) >= 2 * 100000 * 8
