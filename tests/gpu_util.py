@@ -1,4 +1,6 @@
 """Helpers for the GPU parity tests: move a workload to the device and run the C-ABI path on it."""
+import os
+
 import numpy as np
 import torch
 
@@ -33,6 +35,7 @@ def padded_ldh(H: int) -> int:
 def run_forward(w: wl.Workload, mode=jdb.MODE_AUTO, pad_ld=False, sync_schedule=True, flags=0, tuning=0, to_host=True,
                 bench_ld=False):
     """bench_ld: the leading dimensions the benchmark uses (x rows padded to 8, h/c rows to 4 elements)."""
+    flags |= int(os.environ.get("JDB_TEST_EXTRA_FLAGS", "0"))   # e.g. 2: the whole suite with the kernels' index checks on
     forest, x, packed, precision = device_inputs(w, pad_ld or bench_ld)
     sched = jdb.jdb_schedule(forest, sync=sync_schedule)
     ldh = (w.H + 3) // 4 * 4 if bench_ld else (padded_ldh(w.H) if pad_ld else w.H)
