@@ -208,6 +208,8 @@ size_t jdb_forward_workspace_bytes(int32_t n_nodes, int32_t n_internal_bound, in
  * schedule from jdb_schedule_async), in which case the call synchronises at the end to report
  * JDB_ERR_NOT_A_FOREST / JDB_ERR_TIMEOUT.  With JDB_FLAG_NO_SYNC it does not synchronise either (as long as
  * the level count is known or H <= 192) and those two conditions are reported by jdb_sched_status.
+ * JDB_FP32 with H > 192 and a schedule from jdb_schedule runs level by level through a tiled GEMM and synchronises once, at
+ * its start, to read the level table (with JDB_FLAG_NO_SYNC, an explicit mode or the debug checks: the plain-ALU kernels).
  * A bounded wait that runs out inside one of the per-level launches (which are asynchronous) is likewise
  * visible through jdb_sched_status only.  JDB_BF16 with H > 192 runs one set of launches per level and needs the
  * level count on the host: after jdb_schedule_async the call first synchronises once to read it. */

@@ -254,6 +254,9 @@ jdb_status jdb_pack_weights(const float* W, const float* U, const float* b, int3
 
 size_t jdb_forward_workspace_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D, int32_t H, int32_t precision) {
     size_t bytes = forward_ws_bytes(n_nodes, n_internal_bound, D, H, precision);
+    // fp32 beyond the cooperative kernel's hidden sizes: the level-by-level GEMM path keeps its arrays behind the plain one's
+    if (precision == JDB_FP32 && H > 0 && !small_levels_f32_supported(H))
+        bytes = align_up(bytes, 256) + forward_f32_gemm_ws_bytes(n_nodes, n_internal_bound, H);
     if (precision == JDB_BF16) {
         size_t tc = forward_tc_ws_bytes(n_nodes, n_internal_bound, D, H);
         if (tc > bytes) bytes = tc;
@@ -346,9 +349,18 @@ jdb_status jdb_treelstm_forward(const jdb_forest* forest, const jdb_sched* sched
     JDB_CUDA_TRY(cudaMemsetAsync(sched->meta + META_TIMEOUT, 0, 2 * sizeof(int32_t), st));
     if (a.debug) JDB_CUDA_TRY(cudaMemsetAsync(sched->meta + META_CHECK, 0, 4 * sizeof(int32_t), st));
     const uint64_t tmo = opts->barrier_timeout_ns ? opts->barrier_timeout_ns : 2000000000ull;
+    // fp32 with a hidden size beyond the cooperative kernel, level count known, no special request: level by level through
+    // the tiled GEMM (2.5 times the plain-ALU level loop at H = 512); it reads the level table back, so a caller that
+    // forbids synchronisation, asks for a mode or for the index checks keeps the plain-ALU kernels
+    const bool f32_gemm = !tc && opts->precision == JDB_FP32 && known && opts->mode == JDB_MODE_AUTO && !small_levels_f32_supported(H) &&
+                          !a.debug && !(opts->flags & JDB_FLAG_NO_SYNC);
     if (tc)
         s = forward_tc_enqueue(a, pk + L.total, n_levels_host, n_internal_bound, ws, tc_small, tmo, st);
-    else
+    else if (f32_gemm) {
+        s = forward_f32_gemm_enqueue(a, n_levels_host, n_internal_bound,
+                                     (char*)ws + align_up(forward_ws_bytes(N, n_internal_bound, D, H, opts->precision), 256), st);
+        mode = JDB_MODE_PER_LEVEL;   // nothing cooperative ran: no status to wait for
+    } else
         s = forward_enqueue(a, n_levels_host, n_internal_bound, mode, tmo, st);
     if (s != JDB_OK) return s;
     if (a.debug || (mode == JDB_MODE_PERSISTENT && !(opts->flags & JDB_FLAG_NO_SYNC))) {

@@ -25,15 +25,6 @@ namespace {
 
 constexpr int SWEEP_STEPS = 2;   // least K steps per part when a level's GEMM is split to fill the SMs
 
-// lv[l] = level_ptr[l], lv[L + 1 + l] = edge slots before level l, l = 0 .. L
-__global__ void level_table_kernel(const int32_t* level_ptr, const int* edge_ptr, int n_levels, int* lv) {
-    const int l = blockIdx.x * blockDim.x + threadIdx.x;
-    if (l <= n_levels) {
-        lv[l] = level_ptr[l];
-        lv[n_levels + 1 + l] = edge_ptr[level_ptr[l]];
-    }
-}
-
 // ---- pointwise kernels ----------------------------------------------------------------------------------------------
 
 // dH = grad_h, dC = grad_c (or 0): the running gradients of every node's state

@@ -246,6 +246,32 @@ __global__ void nary_pointwise_kernel(const int32_t* __restrict__ perm, const in
     }
 }
 
+// The Child-Sum cell's pointwise part on the packed fp32 layout (columns interleaved by gate: hidden unit j, gate g at
+// 4 j + g): Z rows hold W x + b, T rows (absent for leaves) h~ U^T of which the forget column is not used, FE rows U_f h_k.
+__global__ void childsum_pointwise_il_kernel(const int32_t* __restrict__ perm, const int* __restrict__ edge_ptr,
+                                             const int* __restrict__ slot_child, int lo, int m, int H, const float* __restrict__ Z,
+                                             const float* __restrict__ T, const float* __restrict__ FE, float* __restrict__ h,
+                                             float* __restrict__ c, long long ldh) {
+    const int r = blockIdx.x * blockDim.y + threadIdx.y;
+    if (r >= m) return;
+    const int j = perm[lo + r];
+    const int s0 = edge_ptr[lo + r], s1 = edge_ptr[lo + r + 1];
+    const float4* z = reinterpret_cast<const float4*>(Z + (long long)r * 4 * H);
+    const float4* t = T ? reinterpret_cast<const float4*>(T + (long long)r * 4 * H) : nullptr;
+    for (int col = threadIdx.x; col < H; col += blockDim.x) {
+        float4 g = z[col];
+        if (t) {
+            const float4 u = t[col];
+            g.x += u.x; g.y += u.y; g.z += u.z;
+        }
+        float cc = sigmoidf_(g.x) * tanhf(g.z);
+        for (int s = s0; s < s1; ++s)
+            cc += sigmoidf_(g.w + FE[(long long)s * H + col]) * c[(long long)slot_child[s] * ldh + col];
+        c[(long long)j * ldh + col] = cc;
+        h[(long long)j * ldh + col] = sigmoidf_(g.y) * tanhf(cc);
+    }
+}
+
 struct PlanWorkspace {
     int32_t *comp, *tmp0, *tmp1, *hist;
     int *block_sum, *flags;   // flags[0] slot count, flags[1] bad key
@@ -296,6 +322,93 @@ CellsWorkspace carve_cells(void* ws, long long n, long long e, int H, int amax, 
 }
 
 }  // namespace
+
+// ---- fp32 forward of the Child-Sum cell for hidden sizes beyond the cooperative kernel (forward_simt.cu calls this) ----
+struct F32Workspace {
+    float *Z, *T, *HS, *FE;
+    int *edge_ptr, *slot_child, *slot_ppos, *block_sum, *lv;
+    size_t total;
+};
+static F32Workspace carve_f32(void* ws, long long n, long long ni, int H) {
+    F32Workspace w{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return (char*)ws + o; };
+    w.Z = (float*)take((size_t)n * 4 * H * sizeof(float));
+    w.T = (float*)take((size_t)ni * 4 * H * sizeof(float));
+    w.HS = (float*)take((size_t)ni * H * sizeof(float));
+    w.FE = (float*)take((size_t)n * H * sizeof(float));      // a forest has fewer edges than nodes
+    w.edge_ptr = (int*)take((size_t)(n + 1) * sizeof(int));
+    w.slot_child = (int*)take((size_t)n * sizeof(int));
+    w.slot_ppos = (int*)take((size_t)n * sizeof(int));
+    w.block_sum = (int*)take((size_t)(n / SCAN_BLOCK + 2) * sizeof(int));
+    w.lv = (int*)take((size_t)(2 * (n + 2)) * sizeof(int));
+    w.total = off;
+    return w;
+}
+
+size_t forward_f32_gemm_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t H) {
+    return carve_f32(nullptr, n_nodes > 0 ? n_nodes : 1, n_internal_bound > 0 ? n_internal_bound : 1, H).total;
+}
+
+// Level by level through the tiled fp32 GEMM: W x + b of the level's rows, h~ U^T, U_f h_k over the level's edge slots,
+// then the pointwise part.  Needs the level table on the host: copies it back and synchronises `st` once.
+jdb_status forward_f32_gemm_enqueue(const ForwardArgs& a, int n_levels, int n_internal_bound, void* ws, cudaStream_t st) {
+    const int n = a.n_nodes, ne = a.n_edges, H = a.H, D = a.D, L = n_levels;
+    if (n <= 0 || L <= 0) return JDB_OK;
+    DevInfo* di = dev_info();
+    if (!di) return JDB_ERR_CUDA;
+    const int n_sm = di->n_sm;
+    F32Workspace w = carve_f32(ws, n, n_internal_bound > 0 ? n_internal_bound : 1, H);
+    const int32_t* perm = a.perm;
+    const int sb = n / SCAN_BLOCK + 1;
+    slot_count_kernel<<<sb, SCAN_BLOCK, 0, st>>>(a.child_ptr, perm, n, w.block_sum);
+    block_sums_scan_kernel<<<1, SCAN_BLOCK, 0, st>>>(w.block_sum, sb);
+    slot_fill_kernel<<<sb, SCAN_BLOCK, 0, st>>>(a.child_ptr, a.child_idx, perm, n, ne, w.block_sum, w.edge_ptr, w.slot_child, w.slot_ppos);
+    level_table_kernel<<<ceil_div(L + 1, 256), 256, 0, st>>>(a.level_ptr, w.edge_ptr, L, w.lv);
+    JDB_CUDA_TRY(cudaGetLastError());
+    std::vector<int> lv(2 * (size_t)(L + 1));
+    JDB_CUDA_TRY(cudaMemcpyAsync(lv.data(), w.lv, lv.size() * sizeof(int), cudaMemcpyDeviceToHost, st));
+    JDB_CUDA_TRY(cudaStreamSynchronize(st));
+    const int* lp = lv.data();
+    const int* eo = lv.data() + (L + 1);
+    if (lp[0] != 0 || lp[L] != n || eo[L] != ne || n - lp[1] > n_internal_bound) return JDB_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l)
+        if (lp[l + 1] < lp[l] || eo[l + 1] < eo[l]) return JDB_ERR_INVALID_ARG;
+
+    if (a.ev_begin) JDB_CUDA_TRY(cudaEventRecord(a.ev_begin, st));
+    const dim3 pw_block(H >= 128 ? 128 : (H > 32 ? 64 : 32), H >= 128 ? 2 : (H > 32 ? 4 : 8));
+    jdb_status r;
+    for (int l = 0; l < L; ++l) {
+        const int lo = lp[l], m = lp[l + 1] - lp[l];
+        if (m <= 0) continue;
+        {   // Z = x[rows] Wt + bias (columns interleaved by gate, as the packed weights are)
+            GemmArgs g{};
+            g.A = (const float*)a.x; g.lda = a.ldx; g.a_idx = perm + lo; g.B = a.Wt; g.ldb = 4LL * H; g.C = w.Z; g.ldc = 4LL * H;
+            g.M = m; g.N = 4 * H; g.K = D; g.bias = a.bias;
+            if ((r = gemm<true, true>(g, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
+        }
+        const int e0 = eo[l], e1 = eo[l + 1];
+        if (l > 0) {
+            child_sum_f32_kernel<<<ceil_div(m, pw_block.y), pw_block, 0, st>>>(a.child_ptr, a.child_idx, perm, lo, m, H, a.h, a.ldh, w.HS);
+            GemmArgs g{};
+            g.A = w.HS; g.lda = H; g.B = a.Ut; g.ldb = 4LL * H; g.C = w.T; g.ldc = 4LL * H; g.M = m; g.N = 4 * H; g.K = H;
+            if ((r = gemm<true, true>(g, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
+            if (e1 > e0) {
+                GemmArgs f{};
+                f.A = a.h; f.lda = a.ldh; f.a_idx = w.slot_child + e0; f.B = a.Uft; f.ldb = H; f.C = w.FE + (size_t)e0 * H; f.ldc = H;
+                f.M = e1 - e0; f.N = H; f.K = H;
+                if ((r = gemm<true, true>(f, SLOT_STEPS, n_sm, st)) != JDB_OK) return r;
+            }
+        }
+        childsum_pointwise_il_kernel<<<ceil_div(m, pw_block.y), pw_block, 0, st>>>(perm, w.edge_ptr, w.slot_child, lo, m, H, w.Z,
+                                                                                   l > 0 ? w.T : nullptr, w.FE, a.h, a.c, a.ldh);
+        JDB_CUDA_TRY(cudaGetLastError());
+        if (l == 0 && a.ev_xproj_done) JDB_CUDA_TRY(cudaEventRecord(a.ev_xproj_done, st));   // the leaves: projection only
+    }
+    if (a.ev_levels_done) JDB_CUDA_TRY(cudaEventRecord(a.ev_levels_done, st));
+    return JDB_OK;
+}
+
 }  // namespace jdb
 
 using namespace jdb;

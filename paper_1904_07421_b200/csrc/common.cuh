@@ -151,6 +151,12 @@ size_t forward_tc_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t D,
 jdb_status forward_tc_enqueue(const ForwardArgs& fa, const void* packed_tc, int n_levels, int n_internal_bound,
                               void* ws, bool use_small, uint64_t timeout_ns, cudaStream_t st);
 
+// ---- batcher.cu ------------------------------------------------------------------------------
+// fp32 forward through the tiled GEMM for hidden sizes the cooperative fp32 kernel does not hold; needs the level count
+// on the host and synchronises once for the level table
+size_t forward_f32_gemm_ws_bytes(int32_t n_nodes, int32_t n_internal_bound, int32_t H);
+jdb_status forward_f32_gemm_enqueue(const ForwardArgs& a, int n_levels, int n_internal_bound, void* ws, cudaStream_t st);
+
 // ---- api.cu ----------------------------------------------------------------------------------
 // one request from host buffers: enqueue everything on `stream` (copies in, analysis, forward, copies back) without
 // waiting, and read the recorded status once the stream has drained

@@ -92,6 +92,15 @@ __global__ void __launch_bounds__(SCAN_BLOCK) slot_fill_kernel(const int32_t* ch
     }
 }
 
+// lv[l] = level_ptr[l], lv[L + 1 + l] = edge slots before level l, l = 0 .. L
+__global__ void level_table_kernel(const int32_t* level_ptr, const int* edge_ptr, int n_levels, int* lv) {
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l <= n_levels) {
+        lv[l] = level_ptr[l];
+        lv[n_levels + 1 + l] = edge_ptr[level_ptr[l]];
+    }
+}
+
 // HS[r] = sum of the children's h of the internal node at position n_leaves + r (child-list order)
 __global__ void child_sum_f32_kernel(const int32_t* __restrict__ child_ptr, const int32_t* __restrict__ child_idx,
                                      const int32_t* __restrict__ perm, int n_leaves, int n_int, int H,

@@ -534,3 +534,20 @@ def test_tree_partitioned_cooperative_loop_agrees_bit_for_bit_with_grid_barriers
         h1, c1, _ = run_forward(w, pad_ld=True, tuning=jdb.TUNE_SET | jdb.TUNE_TREE_GROUPS)
         assert np.array_equal(h0, h1) and np.array_equal(c0, c1)
         check(w, h1, c1, TOL_BF16_MATCHED, quantize=matched(w))
+
+
+@pytest.mark.parametrize("D,H", [(40, 200), (97, 257), (64, 512)])
+def test_fp32_large_hidden_size_runs_through_the_gemm_levels(D, H):
+    """fp32 with H > 192 and a synchronised schedule goes level by level through the tiled GEMM; the same call with
+    JDB_FLAG_NO_SYNC keeps the plain-ALU cooperative kernel.  Both against the checker (1e-4) and against each other."""
+    parents = [[-1, 0, 0, 1, 1, 1, 2, 5, 5, 5, 5], [-1] + [0] * 140, [-1, 0, 1, 2, 3], [-1], [-1] + list(range(20))] * 12
+    w = wl.make_custom(parents, D=D, H=H, seed=900 + H, precision="fp32", bias="random")
+    g, new_id = wl.relabel(w.forest, np.random.default_rng(4))
+    tok = np.empty_like(w.token)
+    tok[new_id] = w.token
+    w.forest, w.token = g, tok
+    h0, c0, _ = run_forward(w, pad_ld=True)
+    check(w, h0, c0, TOL_FP32)
+    h1, c1, s = run_forward(w, pad_ld=True, flags=jdb.FLAG_NO_SYNC)
+    assert jdb.jdb_sched_status(s)[0] > 0
+    assert np.max(np.abs(h0 - h1)) <= 2e-5 and np.max(np.abs(c0 - c1)) <= 2e-5
