@@ -301,7 +301,7 @@ size_t jdb_batch_plan_workspace_bytes(int32_t n_nodes);
 jdb_status jdb_batch_plan(const jdb_forest *forest, const jdb_sched *sched, const int32_t *key, int32_t n_keys,
                           jdb_plan *out, void *ws, size_t ws_bytes, void *stream);
 
-/* One kind of cell with its own parameters (the "same parameterisation" condition of Section 1: nodes batch only with
+/* One kind of cell with its own parameters (Section 1 lets nodes share a batch only if they also share their parameters: nodes batch only with
  * nodes of the same cell).  W [4H, D], b [4H] in row blocks (i, o, u, f), fp32 row-major device arrays.
  * JDB_CELL_CHILDSUM: the cell of jdb_treelstm_forward, U [4H, H], any number of children.
  * JDB_CELL_NARY: the N-ary Tree-LSTM cell of the same cited model, one recurrent matrix per child position:
