@@ -544,11 +544,32 @@ def time_training(idx: int, w: wl.Workload, device, flush, steps: int = 5, warmu
             fwd.append(e[0].elapsed_time(e[1]))
             bwd.append(e[1].elapsed_time(e[2]))
     tf, tb = statistics.median(fwd), statistics.median(bwd)
+    # mixed precision: the tensor-core forward (bf16 operands) feeding the same fp32 backward pass
+    tf16 = None
+    if w.precision == "bf16":
+        packed16 = jdb.jdb_pack_weights(W, U, b, jdb.BF16)
+        x16 = x.to(torch.bfloat16)
+        fws16 = jdb.forward_workspace(forest, sched, D, H, jdb.BF16)
+        f16 = []
+        for it in range(warmup + steps):
+            flush.add_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            jdb.jdb_schedule(forest, sched, sws)
+            jdb.jdb_treelstm_forward(forest, sched, x16, packed16, D, H, jdb.BF16, h=h, c=c, ws=fws16)
+            e1.record()
+            e1.synchronize()
+            if it >= warmup:
+                f16.append(e0.elapsed_time(e1))
+        tf16 = statistics.median(f16)
+        del packed16, x16, fws16
     flops_b = 3.0 * (8.0 * f.n_nodes * D * H + 6.0 * n_int * H * H + 2.0 * f.n_edges * H * H)
     return {"config": idx, "workload": w.name, "nodes": f.n_nodes, "trees": f.n_trees, "D": D, "H": H, "dtype": "f32",
             "step": "jdb_schedule + jdb_treelstm_forward + jdb_treelstm_backward (loss on the roots)",
             "forward_ms": tf, "backward_ms": tb, "nodes_per_s": f.n_nodes / ((tf + tb) * 1e-3),
-            "trees_per_s": f.n_trees / ((tf + tb) * 1e-3), "backward_flops": flops_b,
+            "trees_per_s": f.n_trees / ((tf + tb) * 1e-3),
+            "forward_bf16_ms": tf16, "trees_per_s_bf16_forward": (f.n_trees / ((tf16 + tb) * 1e-3)) if tf16 else None,
+            "backward_flops": flops_b,
             "backward_tflops": flops_b / (tb * 1e-3) / 1e12,
             "backward_frac_of_fp32_alu_peak": flops_b / (tb * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
             "launches_backward": 4 + 2 + 3 + 3 * max(sched.n_levels - 1, 0) + 1 + 5}
